@@ -1,0 +1,254 @@
+/*
+ * fp64 CPU oracle for the three memory-bound LLM-serving operations of the
+ * Astra paper (Table 1): fused_add_rmsnorm, silu_and_mul, merge_attn_states_lse.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition the CUDA
+ * library is checked against.  It shares no code, header, table or constant
+ * with the CUDA path, and nothing on the product path may call it.
+ *
+ * Every function is the printed formula evaluated in double precision on the
+ * exact values of the 16-bit storage patterns the GPU receives.  No blocking,
+ * fusion or reordering: one loop per index of the formula.  The only
+ * parallelism is an OpenMP "parallel for" over independent rows, used when the
+ * oracle is timed as a CPU baseline (nthreads > 1); it does not change any
+ * arithmetic because rows never interact.
+ *
+ * Storage formats.  dtype 0 = bfloat16 (1 sign, 8 exponent, 7 fraction bits),
+ * dtype 1 = IEEE binary16 (1, 5, 10).  Both are widened exactly to double and
+ * rounded back with round-to-nearest-even, written out arithmetically below
+ * (frexp / ldexp / nearbyint), not with bit tricks, so they can be read against
+ * the format definitions.
+ *
+ * Pins (tests, CPU only): closed forms, invariants, textbook reductions
+ * (plain RMSNorm, two-way softmax, attention over a split key set), library
+ * routines of torch on CPU in fp64, an integer-only bf16 adder for the
+ * residual sum, and torch's own float->bf16 / float->fp16 casts for the
+ * rounding helpers.  No function here is "parity unpinned".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#define ORACLE_BF16 0
+#define ORACLE_FP16 1
+
+typedef struct {
+    int frac_bits; /* explicit fraction bits            */
+    int exp_bits;  /* exponent field width              */
+    int bias;      /* exponent bias                     */
+} storage_format;
+
+static storage_format format_of(int dtype)
+{
+    storage_format f;
+    if (dtype == ORACLE_FP16) {
+        f.frac_bits = 10; f.exp_bits = 5; f.bias = 15;
+    } else {
+        f.frac_bits = 7;  f.exp_bits = 8; f.bias = 127;
+    }
+    return f;
+}
+
+/* Exact value of a 16-bit storage pattern. */
+static double widen(uint16_t bits, storage_format f)
+{
+    int sign = (bits >> 15) & 1;
+    int exp_field = (bits >> f.frac_bits) & ((1 << f.exp_bits) - 1);
+    int frac = bits & ((1 << f.frac_bits) - 1);
+    int exp_all_ones = (1 << f.exp_bits) - 1;
+    double v;
+    if (exp_field == exp_all_ones) {
+        v = frac ? NAN : INFINITY;
+    } else if (exp_field == 0) {
+        /* subnormal: frac * 2^(1 - bias - frac_bits) */
+        v = ldexp((double)frac, 1 - f.bias - f.frac_bits);
+    } else {
+        v = ldexp((double)((1 << f.frac_bits) + frac), exp_field - f.bias - f.frac_bits);
+    }
+    return sign ? -v : v;
+}
+
+/* Round a double to the storage format, nearest-even, return the bit pattern.
+   nearbyint() rounds to nearest-even in the default rounding mode. */
+static uint16_t round_to_storage(double v, storage_format f)
+{
+    uint16_t sign = signbit(v) ? 0x8000u : 0u;
+    int exp_all_ones = (1 << f.exp_bits) - 1;
+    double a = fabs(v);
+    if (isnan(v))
+        return (uint16_t)(sign | (exp_all_ones << f.frac_bits) | (1 << (f.frac_bits - 1)));
+    if (isinf(v))
+        return (uint16_t)(sign | (exp_all_ones << f.frac_bits));
+    if (a == 0.0)
+        return sign;
+
+    int e_min = 1 - f.bias;                 /* exponent of the smallest normal   */
+    int e_max = exp_all_ones - 1 - f.bias;  /* exponent of the largest finite    */
+    int e;
+    (void)frexp(a, &e);                     /* a = m * 2^e, m in [0.5, 1)        */
+    int E = e - 1;                          /* a in [2^E, 2^(E+1))               */
+    if (E < e_min) E = e_min;               /* subnormals share the quantum of e_min */
+    double quantum = ldexp(1.0, E - f.frac_bits);
+    double q = nearbyint(a / quantum);      /* division by a power of two: exact */
+    double r = q * quantum;                 /* the rounded magnitude             */
+
+    /* r may have carried into the next binade; re-derive its exponent. */
+    if (r >= ldexp(1.0, e_max + 1))
+        return (uint16_t)(sign | (exp_all_ones << f.frac_bits)); /* overflow -> inf */
+    if (r < ldexp(1.0, e_min)) {
+        /* subnormal or zero: fraction field counts quanta of 2^(e_min - frac_bits) */
+        uint16_t frac = (uint16_t)(r / ldexp(1.0, e_min - f.frac_bits));
+        return (uint16_t)(sign | frac);
+    }
+    (void)frexp(r, &e);
+    E = e - 1;
+    uint16_t exp_field = (uint16_t)(E + f.bias);
+    uint16_t frac = (uint16_t)(r / ldexp(1.0, E - f.frac_bits) - (double)(1 << f.frac_bits));
+    return (uint16_t)(sign | (exp_field << f.frac_bits) | frac);
+}
+
+/* Exposed so the tests can pin the two helpers on their own. */
+double oracle_widen(uint16_t bits, int dtype)
+{
+    return widen(bits, format_of(dtype));
+}
+
+uint16_t oracle_round_to_storage(double v, int dtype)
+{
+    return round_to_storage(v, format_of(dtype));
+}
+
+/*
+ * fused_add_rmsnorm  (Table 1, Kernel 2):
+ *     y = (x + r) / sqrt( (1/H) * ||x + r||^2 + eps )  (.)  w
+ *
+ * x, r : [T, H] storage patterns.  w : [H].
+ * y_out        : [T, H] doubles, the formula's value.
+ * residual_out : [T, H] storage patterns of the updated residual.
+ *
+ * Readings where Table 1 is silent:
+ *  - The sum s = x + r is formed as a binary32 add (the exact double sum
+ *    rounded once to float).  The updated residual is that float rounded once
+ *    to the storage dtype.  This output is compared bit for bit.
+ *  - The norm uses the float sum itself, not the storage-rounded residual.
+ *  - eps is a float argument taken at its exact value; it sits inside the
+ *    square root, added to the mean of squares, as printed.
+ *  - No rounding between the normalisation and the multiplication by w.
+ */
+void oracle_fused_add_rmsnorm(const uint16_t *x, const uint16_t *r, const uint16_t *w,
+                              int64_t T, int64_t H, float eps, int dtype,
+                              double *y_out, uint16_t *residual_out, int nthreads)
+{
+    storage_format f = format_of(dtype);
+    if (nthreads < 1) nthreads = 1;
+#pragma omp parallel for num_threads(nthreads) schedule(static)
+    for (int64_t t = 0; t < T; ++t) {
+        const uint16_t *xt = x + t * H;
+        const uint16_t *rt = r + t * H;
+        double sum_sq = 0.0;
+        for (int64_t j = 0; j < H; ++j) {
+            double s_exact = widen(xt[j], f) + widen(rt[j], f); /* exact in double */
+            double s = (double)(float)s_exact;                  /* binary32 add    */
+            sum_sq += s * s;
+        }
+        double denom = sqrt(sum_sq / (double)H + (double)eps);
+        for (int64_t j = 0; j < H; ++j) {
+            double s_exact = widen(xt[j], f) + widen(rt[j], f);
+            float s32 = (float)s_exact;
+            residual_out[t * H + j] = round_to_storage((double)s32, f);
+            y_out[t * H + j] = (double)s32 / denom * widen(w[j], f);
+        }
+    }
+}
+
+/*
+ * silu_and_mul  (Table 1, Kernel 3):
+ *     out = SiLU(a) (.) b,   SiLU(z) = z / (1 + e^{-z})
+ *
+ * input : [T, 2*D]; columns 0..D-1 are the gate a, columns D..2D-1 are b.
+ * out   : [T, D] doubles.
+ *
+ * For z below -700, e^{-z} overflows a double; the algebraically identical form
+ * z * e^{z} / (1 + e^{z}) is used there so the function stays total.
+ */
+static double silu(double z)
+{
+    if (z < -700.0) {
+        double ez = exp(z);
+        return z * ez / (1.0 + ez);
+    }
+    return z / (1.0 + exp(-z));
+}
+
+void oracle_silu_and_mul(const uint16_t *input, int64_t T, int64_t D, int dtype,
+                         double *out, int nthreads)
+{
+    storage_format f = format_of(dtype);
+    if (nthreads < 1) nthreads = 1;
+#pragma omp parallel for num_threads(nthreads) schedule(static)
+    for (int64_t t = 0; t < T; ++t) {
+        const uint16_t *row = input + t * 2 * D;
+        for (int64_t i = 0; i < D; ++i) {
+            double a = widen(row[i], f);
+            double b = widen(row[D + i], f);
+            out[t * D + i] = silu(a) * b;
+        }
+    }
+}
+
+/*
+ * merge_attn_states_lse  (Table 1, Kernel 1):
+ *     V_out = (e^{Sa} Va + e^{Sb} Vb) / (e^{Sa} + e^{Sb})
+ *     S_out = log(e^{Sa} + e^{Sb})                        (natural log)
+ *
+ * v_a, v_b : [T, Hh, D] storage patterns.  lse_a, lse_b : [T, Hh] binary32.
+ * v_out    : [T, Hh, D] doubles.           lse_out      : [T, Hh] doubles.
+ *
+ * Evaluated after factoring e^{m}, m = max(Sa, Sb), out of numerator and
+ * denominator; this is the same real number and keeps e^{S} inside double range.
+ *
+ * Readings where Table 1 is silent:
+ *  - One score -inf: its weight is exactly 0 and that side's V does not
+ *    contribute (it is skipped, not multiplied), so the other state is returned.
+ *  - Both scores -inf (an empty state merged with an empty state):
+ *    V_out = 0 and S_out = -inf.
+ *  - +inf or NaN scores are outside the operation's domain: NaN out.
+ */
+void oracle_merge_attn_states_lse(const uint16_t *v_a, const float *lse_a,
+                                  const uint16_t *v_b, const float *lse_b,
+                                  int64_t T, int64_t Hh, int64_t D, int dtype,
+                                  double *v_out, double *lse_out, int nthreads)
+{
+    storage_format f = format_of(dtype);
+    if (nthreads < 1) nthreads = 1;
+#pragma omp parallel for num_threads(nthreads) schedule(static)
+    for (int64_t th = 0; th < T * Hh; ++th) {
+        double sa = (double)lse_a[th];
+        double sb = (double)lse_b[th];
+        const uint16_t *va = v_a + th * D;
+        const uint16_t *vb = v_b + th * D;
+        double *vo = v_out + th * D;
+
+        if (isnan(sa) || isnan(sb) || sa == INFINITY || sb == INFINITY) {
+            for (int64_t d = 0; d < D; ++d) vo[d] = NAN;
+            lse_out[th] = NAN;
+            continue;
+        }
+        if (sa == -INFINITY && sb == -INFINITY) {
+            for (int64_t d = 0; d < D; ++d) vo[d] = 0.0;
+            lse_out[th] = -INFINITY;
+            continue;
+        }
+        double m = sa > sb ? sa : sb;
+        double wa = exp(sa - m); /* exp(-inf) = 0 exactly */
+        double wb = exp(sb - m);
+        double denom = wa + wb;
+        for (int64_t d = 0; d < D; ++d) {
+            double num = 0.0;
+            if (wa != 0.0) num += wa * widen(va[d], f);
+            if (wb != 0.0) num += wb * widen(vb[d], f);
+            vo[d] = num / denom;
+        }
+        lse_out[th] = m + log(denom);
+    }
+}
