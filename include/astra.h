@@ -1,0 +1,104 @@
+/*
+ * astra.h -- C ABI of the B200 (sm_100a) library for the three memory-bound LLM-serving
+ * operations studied in "Astra: A Multi-Agent System for GPU Kernel Performance Optimization"
+ * (Table 1: merge_attn_states_lse, fused_add_rmsnorm, silu_and_mul).
+ *
+ * Conventions shared by every entry point
+ *   - Every data pointer is a DEVICE pointer on the current CUDA device, owned by the caller.
+ *     The library allocates nothing, keeps no state between calls, and never synchronises:
+ *     work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream)
+ *     and the call returns immediately.  Host pointers are not detected (undefined behaviour).
+ *   - Tensors are dense and row-major (the last index is contiguous; a row's pitch is its width).
+ *   - `dtype` selects the 16-bit storage type of all value tensors of the call.  Arithmetic is
+ *     binary32 throughout, with a single round-to-nearest-even to the storage type at each store.
+ *   - Pointers need only the natural alignment of their element (2 bytes for values, 4 for
+ *     scores).  Wider alignment is detected and exploited inside; widths need not be multiples
+ *     of 8.  A pointer with less than element alignment gives ASTRA_ERR_MISALIGNED.
+ *   - Errors are return codes only: nothing is printed, thrown or aborted, and on any error
+ *     nothing has been launched.  A zero-sized first dimension (T == 0) is ASTRA_OK and launches
+ *     nothing; any other non-positive extent is ASTRA_ERR_BAD_SHAPE.
+ *   - Non-finite inputs never trap; they propagate by IEEE rules except where stated below.
+ */
+#ifndef ASTRA_H_
+#define ASTRA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ASTRA_BF16 = 0, /* bfloat16: 1 sign, 8 exponent, 7 fraction bits */
+    ASTRA_FP16 = 1  /* IEEE binary16                                  */
+} astra_dtype_t;
+
+typedef enum {
+    ASTRA_OK = 0,
+    ASTRA_ERR_NULL_POINTER = 1, /* a required pointer is NULL                         */
+    ASTRA_ERR_BAD_SHAPE = 2,    /* an extent is negative, zero where not allowed, or too large */
+    ASTRA_ERR_BAD_DTYPE = 3,    /* dtype is not one of astra_dtype_t                  */
+    ASTRA_ERR_MISALIGNED = 4,   /* a pointer is not aligned to its element size       */
+    ASTRA_ERR_CUDA = 5,         /* the CUDA runtime reported an error at launch       */
+    ASTRA_ERR_OVERLAP = 6       /* an output overlaps an input in a way not allowed   */
+} astra_status_t;
+
+/*
+ * fused_add_rmsnorm (Table 1, Kernel 2):
+ *     y = (x + r) / sqrt( (1/H) * ||x + r||_2^2 + eps )  (.)  w         per row of H elements
+ *
+ *   x        [T, H]  in: x.          out: y                       (updated in place)
+ *   residual [T, H]  in: r.          out: x + r                   (updated in place)
+ *   weight   [H]     in: w.
+ *   eps      added to the mean of squares, inside the square root.
+ *
+ * The sum x + r is one binary32 addition.  `residual` receives that sum rounded once to the
+ * storage type (bit-exact, independent of launch shape).  The norm is taken over the unrounded
+ * binary32 sums, and nothing is rounded between the normalisation and the multiplication by w.
+ * x and residual must not overlap each other or weight.
+ */
+astra_status_t astra_fused_add_rmsnorm(void *x, void *residual, const void *weight,
+                                       int64_t T, int64_t H, float eps,
+                                       astra_dtype_t dtype, void *cuda_stream);
+
+/*
+ * silu_and_mul (Table 1, Kernel 3):
+ *     out = SiLU(a) (.) b,   SiLU(z) = z / (1 + e^{-z})
+ *
+ *   input [T, 2*D]  in: each row is [ a (D gate values) | b (D up values) ].
+ *   out   [T, D]    out.  Must not overlap input (checked: ASTRA_ERR_OVERLAP).
+ *
+ * SiLU(a) is not rounded to the storage type before the multiplication by b.
+ */
+astra_status_t astra_silu_and_mul(void *out, const void *input, int64_t T, int64_t D,
+                                  astra_dtype_t dtype, void *cuda_stream);
+
+/*
+ * merge_attn_states_lse (Table 1, Kernel 1): merge two partial attention results, each given
+ * as an output vector and the natural-log sum of exponentials of its logits.
+ *     V_out = (e^{Sa} Va + e^{Sb} Vb) / (e^{Sa} + e^{Sb})
+ *     S_out = log(e^{Sa} + e^{Sb})
+ *
+ *   v_a, v_b  [T, Hh, D]  in.        lse_a, lse_b  [T, Hh] binary32, in.
+ *   v_out     [T, Hh, D]  out.       lse_out       [T, Hh] binary32, out; may be NULL (not written).
+ *
+ * The two weights are computed once per (token, head).  v_out may be exactly v_a or v_b
+ * (in-place merge of the values); any other overlap of v_out with an input, and any overlap of
+ * lse_out with lse_a or lse_b, gives ASTRA_ERR_OVERLAP.
+ * A score of -inf denotes an empty state: its weight is exactly 0, its V is ignored (even if
+ * not finite), and the other state is returned unchanged.  If both scores are -inf the result
+ * is V_out = 0, S_out = -inf.  A score of +inf or NaN is outside the domain: NaN is produced.
+ */
+astra_status_t astra_merge_attn_states_lse(void *v_out, float *lse_out,
+                                           const void *v_a, const float *lse_a,
+                                           const void *v_b, const float *lse_b,
+                                           int64_t T, int64_t Hh, int64_t D,
+                                           astra_dtype_t dtype, void *cuda_stream);
+
+/* Static, NUL-terminated description of a status code (never NULL). */
+const char *astra_status_string(astra_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASTRA_H_ */

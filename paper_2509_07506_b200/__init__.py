@@ -1,0 +1,14 @@
+"""B200 (sm_100a) kernels for fused_add_rmsnorm, silu_and_mul and merge_attn_states_lse.
+
+``binding`` holds the Python side of the C ABI declared in ``include/astra.h``; ``workloads`` the
+seeded synthetic inputs; ``build`` compiles the shared library.  Importing the package does not
+load the library; the first call does, and fails loudly if it has not been built.
+"""
+from .binding import (  # noqa: F401
+    AstraError,
+    astra_fused_add_rmsnorm,
+    astra_merge_attn_states_lse,
+    astra_silu_and_mul,
+    load_library,
+    status_string,
+)

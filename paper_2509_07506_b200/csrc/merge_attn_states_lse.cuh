@@ -1,0 +1,92 @@
+// merge_attn_states_lse (Astra paper, Table 1, Kernel 1):
+//     V_out = (e^{Sa} Va + e^{Sb} Vb) / (e^{Sa} + e^{Sb}),   S_out = log(e^{Sa} + e^{Sb}).
+//
+// HBM-bound: per (token, head) row of D elements, 2*D*2 bytes are read and D*2 written, plus three
+// 4-byte scores.  The two mixing weights depend only on the row, so each thread derives them once
+// for the vector(s) it owns (the paper's hoisting of the exponentials out of the element loop); the
+// element work is one multiply and one fused multiply-add.
+#pragma once
+
+#include "vec.cuh"
+
+namespace astra {
+
+struct MergeWeights {
+    float wa, wb;   // normalised weights of the two states
+    float lse;      // merged score
+    bool use_a, use_b;
+};
+
+// m = max(Sa, Sb); with t = e^{min - max} in [0, 1]: weight of the larger = 1/(1+t), of the
+// smaller = t/(1+t), S_out = m + log(1+t).  A score of -inf gives t = 0 exactly, so the other state
+// passes through with weight exactly 1; its own V is not used at all.  Both -inf: empty result.
+__device__ __forceinline__ MergeWeights merge_weights(float sa, float sb) {
+    MergeWeights r;
+    const float m = fmaxf(sa, sb);
+    const float lo = fminf(sa, sb);
+    if (m == -INFINITY) {  // both states empty
+        r.wa = 0.f; r.wb = 0.f; r.lse = -INFINITY; r.use_a = false; r.use_b = false;
+        return r;
+    }
+    // t in [0, 1]; exactly 0 for lo = -inf, exactly 1 for lo = m.  Non-flushing ex2, so a weight
+    // below 2^-126 is still a (subnormal) weight rather than zero.
+    float t;
+    asm("ex2.approx.f32 %0, %1;" : "=f"(t) : "f"((lo - m) * 1.4426950408889634f));
+    const float inv = __fdividef(1.0f, 1.0f + t);
+    const float w_hi = inv, w_lo = t * inv;
+    const bool a_is_hi = sa >= sb;
+    r.wa = a_is_hi ? w_hi : w_lo;
+    r.wb = a_is_hi ? w_lo : w_hi;
+    r.lse = m + log1pf(t);
+    // +inf or NaN scores are outside the domain (e^{S} / e^{S} = inf / inf): everything becomes NaN.
+    if (!(m < INFINITY) || sa != sa || sb != sb) { r.wa = r.wb = r.lse = __int_as_float(0x7fc00000); }
+    r.use_a = !(r.wa == 0.f);
+    r.use_b = !(r.wb == 0.f);
+    return r;
+}
+
+// Flat indexing over vectors of VEC elements: vector v belongs to row = v / nvec (row = token*Hh+head).
+template <int DT, int VEC, int UNROLL, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+merge_attn_states_lse_kernel(uint16_t *v_out, float *lse_out,
+                             const uint16_t *v_a, const float *lse_a,
+                             const uint16_t *v_b, const float *lse_b,
+                             uint32_t total_vecs, FastDiv nvec) {
+    const uint32_t base = blockIdx.x * (THREADS * UNROLL) + threadIdx.x;
+    Pack<VEC> a[UNROLL], b[UNROLL];
+    float sa[UNROLL], sb[UNROLL];
+    uint32_t row[UNROLL];
+#pragma unroll
+    for (int j = 0; j < UNROLL; ++j) {
+        const uint32_t v = base + j * THREADS;
+        if (v < total_vecs) {
+            row[j] = nvec.div(v);
+            // v_out may be exactly v_a or v_b, so these are ordinary (coherent) loads; the thread
+            // that reads a vector is the only one that writes it
+            a[j] = load<VEC, Ld::Stream>(v_a + static_cast<int64_t>(v) * VEC);
+            b[j] = load<VEC, Ld::Stream>(v_b + static_cast<int64_t>(v) * VEC);
+            sa[j] = lse_a[row[j]];
+            sb[j] = lse_b[row[j]];
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < UNROLL; ++j) {
+        const uint32_t v = base + j * THREADS;
+        if (v < total_vecs) {
+            const MergeWeights mw = merge_weights(sa[j], sb[j]);
+            float fa[VEC], fb[VEC], fo[VEC];
+            widen<DT, VEC>(a[j], fa);
+            widen<DT, VEC>(b[j], fb);
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                // a zero-weight side is dropped, not multiplied: its payload may be Inf/NaN garbage
+                const float ta = mw.use_a ? fa[i] * mw.wa : 0.f;
+                fo[i] = mw.use_b ? fmaf(fb[i], mw.wb, ta) : ta;
+            }
+            store<VEC, St::Stream>(v_out + static_cast<int64_t>(v) * VEC, narrow<DT, VEC>(fo));
+            if (lse_out != nullptr && v == row[j] * nvec.d) lse_out[row[j]] = mw.lse;
+        }
+    }
+}
+
+}  // namespace astra

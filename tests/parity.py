@@ -1,0 +1,81 @@
+"""Tolerances and comparison helpers for the GPU-vs-oracle parity tests.
+
+Gates (oracle values are fp64; GPU values are the exact values of its 16-bit outputs):
+  - residual sum: bit-for-bit.
+  - bf16 outputs: |gpu - oracle| <= 2 * ulp_bf16(|oracle|), ulp_bf16(v) = 2^(floor(log2 v) - 7)
+    (floored at the subnormal quantum 2^-133); oracle == 0 requires gpu == +-0.
+  - fp16 outputs: |gpu - oracle| <= max(1e-3, 2 * ulp_fp16(|oracle|)), ulp_fp16(v) = 2^(floor(log2 v) - 10)
+    (floored at 2^-24).  The plain 1e-3 cannot hold above |y| = 4, where half an fp16 ulp already
+    exceeds it; the count of elements beyond the literal 1e-3 is returned for reporting.
+  - merge values: the blend a*Va + b*Vb can cancel, so the binary32 accumulation floor
+    2^-22 * (|a*Va| + |b*Vb|) is added to the gate.
+  - merged score: |gpu - oracle| <= 1e-5; -inf must be -inf.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+BF16, FP16 = 0, 1
+_FRAC = {BF16: 7, FP16: 10}
+_EMIN = {BF16: -126, FP16: -14}
+
+
+def ulp(v: np.ndarray, dtype: int) -> np.ndarray:
+    """Spacing of the storage format at |v| (v != 0 finite); the subnormal quantum below the normals."""
+    a = np.abs(np.asarray(v, dtype=np.float64))
+    with np.errstate(divide="ignore"):
+        e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
+    # guard against log2 rounding at exact powers of two
+    e = np.where(np.ldexp(1.0, e.astype(np.int64)) > a, e - 1, e)
+    e = np.where(np.ldexp(1.0, (e + 1).astype(np.int64)) <= a, e + 1, e)
+    e = np.maximum(e, _EMIN[dtype])
+    return np.ldexp(1.0, (e - _FRAC[dtype]).astype(np.int64))
+
+
+def value_gate(oracle: np.ndarray, dtype: int, extra: np.ndarray | float = 0.0) -> np.ndarray:
+    tol = 2.0 * ulp(oracle, dtype)
+    if dtype == FP16:
+        tol = np.maximum(tol, 1e-3)
+    tol = np.where(oracle == 0.0, 0.0, tol)
+    return tol + extra
+
+
+def check_values(gpu: np.ndarray, oracle: np.ndarray, dtype: int, extra=0.0, what: str = "") -> dict:
+    """Assert the gate elementwise; returns summary statistics."""
+    gpu = np.asarray(gpu, dtype=np.float64)
+    oracle = np.asarray(oracle, dtype=np.float64)
+    assert gpu.shape == oracle.shape, (gpu.shape, oracle.shape)
+    nan_o = np.isnan(oracle)
+    assert np.array_equal(np.isnan(gpu), nan_o), f"{what}: NaN pattern differs"
+    fin = ~nan_o
+    err = np.zeros_like(oracle)
+    with np.errstate(invalid="ignore"):
+        err[fin] = np.where(gpu[fin] == oracle[fin], 0.0, np.abs(gpu[fin] - oracle[fin]))
+    tol = value_gate(np.where(fin, oracle, 1.0), dtype, extra)
+    bad = fin & ~(err <= tol)
+    if bad.any():
+        i = np.flatnonzero(bad)[0]
+        raise AssertionError(
+            f"{what}: {bad.sum()} of {bad.size} elements outside the gate; first at flat index {i}: "
+            f"gpu={gpu.ravel()[i]!r} oracle={oracle.ravel()[i]!r} err={err.ravel()[i]:.3e} "
+            f"tol={np.broadcast_to(tol, oracle.shape).ravel()[i]:.3e}")
+    u = ulp(np.where(fin & (oracle != 0), oracle, 1.0), dtype)
+    return {
+        "max_err_ulp": float(np.max(np.where(fin & (oracle != 0), err / u, 0.0))) if oracle.size else 0.0,
+        "max_abs_err": float(err.max()) if oracle.size else 0.0,
+        "beyond_literal_1e-3": int((err > 1e-3).sum()),
+    }
+
+
+def check_lse(gpu: np.ndarray, oracle: np.ndarray, what: str = "") -> float:
+    gpu = np.asarray(gpu, dtype=np.float64)
+    oracle = np.asarray(oracle, dtype=np.float64)
+    assert gpu.shape == oracle.shape
+    nan_o = np.isnan(oracle)
+    assert np.array_equal(np.isnan(gpu), nan_o), f"{what}: NaN pattern differs"
+    inf_o = np.isinf(oracle)
+    assert np.array_equal(gpu[inf_o], oracle[inf_o]), f"{what}: infinite scores differ"
+    fin = ~(nan_o | inf_o)
+    err = np.abs(gpu[fin] - oracle[fin])
+    assert np.all(err <= 1e-5), f"{what}: max score error {err.max():.3e} > 1e-5"
+    return float(err.max()) if err.size else 0.0

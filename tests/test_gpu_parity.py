@@ -1,0 +1,308 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 oracle, element by element,
+on the same seeded host inputs.  Every device buffer sits between guard regions that are checked
+after each launch.  Gates are defined in parity.py."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2509_07506_b200 as astra
+from paper_2509_07506_b200 import workloads as wl
+from parity import check_lse, check_values
+
+pytestmark = pytest.mark.gpu
+
+BF16, FP16 = wl.BF16, wl.FP16
+GUARD = 512  # bytes on each side of every device buffer
+NCPU = max(1, len(__import__("os").sched_getaffinity(0)))
+
+
+class Guarded:
+    """A device tensor placed `offset_elems` elements past a 256-byte-aligned point, with
+    pattern-filled guard regions before and after it."""
+
+    def __init__(self, host: torch.Tensor, offset_elems: int = 0):
+        host = host.contiguous()
+        self.nbytes = host.numel() * host.element_size()
+        off = offset_elems * host.element_size()
+        self.raw = torch.full((GUARD + off + self.nbytes + GUARD,), 0xA5, dtype=torch.uint8, device="cuda")
+        self.lo = GUARD + off
+        inner = self.raw[self.lo:self.lo + self.nbytes]
+        self.t = inner.view(host.dtype).view(host.shape)
+        self.t.copy_(host)
+
+    def check(self):
+        assert bool((self.raw[:self.lo] == 0xA5).all()), "guard before the buffer was overwritten"
+        assert bool((self.raw[self.lo + self.nbytes:] == 0xA5).all()), "guard after the buffer was overwritten"
+
+    def host(self) -> torch.Tensor:
+        return self.t.cpu()
+
+
+def f64(t: torch.Tensor) -> np.ndarray:
+    return t.to(torch.float64).numpy()
+
+
+# ---------------------------------------------------------------------------------------------
+# runners
+# ---------------------------------------------------------------------------------------------
+
+def run_rmsnorm(inp: wl.RmsnormInputs, rows=None, offset=0, stream=None):
+    """Runs the library on the full input; compares the given rows (all if None)."""
+    gx, gr, gw = Guarded(inp.x, offset), Guarded(inp.residual, offset), Guarded(inp.weight, offset)
+    astra.astra_fused_add_rmsnorm(gx.t, gr.t, gw.t, inp.eps, stream=stream)
+    torch.cuda.synchronize()
+    for g in (gx, gr, gw):
+        g.check()
+    assert torch.equal(gw.host(), inp.weight)
+    y, r = gx.host(), gr.host()
+    if rows is None:
+        rows = np.arange(inp.x.shape[0])
+    rows = np.asarray(rows)
+    if rows.size == 0:
+        return {}
+    idx = torch.from_numpy(rows)
+    oy, orr = oracle.fused_add_rmsnorm(wl.bits(inp.x[idx]), wl.bits(inp.residual[idx]), wl.bits(inp.weight),
+                                       inp.eps, inp.dtype, nthreads=NCPU)
+    assert np.array_equal(wl.bits(r[idx]), orr), "residual sum is not bit-exact"
+    return check_values(f64(y[idx]), oy, inp.dtype, what=f"rmsnorm {tuple(inp.x.shape)}")
+
+
+def run_silu(inp: wl.SiluInputs, rows=None, offset=0):
+    T, twoD = inp.input.shape
+    D = twoD // 2
+    gi = Guarded(inp.input, offset)
+    go = Guarded(torch.zeros((T, D), dtype=inp.input.dtype), offset)
+    astra.astra_silu_and_mul(go.t, gi.t)
+    torch.cuda.synchronize()
+    gi.check(); go.check()
+    assert torch.equal(gi.host(), inp.input)
+    out = go.host()
+    if rows is None:
+        rows = np.arange(T)
+    rows = np.asarray(rows)
+    if rows.size == 0:
+        return {}
+    idx = torch.from_numpy(rows)
+    want = oracle.silu_and_mul(wl.bits(inp.input[idx]), inp.dtype, nthreads=NCPU)
+    return check_values(f64(out[idx]), want, inp.dtype, what=f"silu {tuple(inp.input.shape)}")
+
+
+def run_merge(inp: wl.MergeInputs, tokens=None, offset=0, in_place=None, with_lse=True):
+    T, Hh, D = inp.v_a.shape
+    ga, gb = Guarded(inp.v_a, offset), Guarded(inp.v_b, offset)
+    gsa, gsb = Guarded(inp.lse_a, offset), Guarded(inp.lse_b, offset)
+    if in_place == "a":
+        go = ga
+    elif in_place == "b":
+        go = gb
+    else:
+        go = Guarded(torch.zeros_like(inp.v_a), offset)
+    gso = Guarded(torch.full((T, Hh), 123.0, dtype=torch.float32), offset)
+    astra.astra_merge_attn_states_lse(go.t, gso.t if with_lse else None, ga.t, gsa.t, gb.t, gsb.t)
+    torch.cuda.synchronize()
+    for g in (ga, gb, gsa, gsb, go, gso):
+        g.check()
+    assert torch.equal(gsa.host(), inp.lse_a) and torch.equal(gsb.host(), inp.lse_b)
+    v, s = go.host(), gso.host()
+    if not with_lse:
+        assert bool((s == 123.0).all())
+    if tokens is None:
+        tokens = np.arange(T)
+    tokens = np.asarray(tokens)
+    if tokens.size == 0:
+        return {}
+    idx = torch.from_numpy(tokens)
+    ov, os_ = oracle.merge_attn_states_lse(wl.bits(inp.v_a[idx]), inp.lse_a[idx].numpy(), wl.bits(inp.v_b[idx]),
+                                           inp.lse_b[idx].numpy(), inp.dtype, nthreads=NCPU)
+    # binary32 accumulation floor of the two-term blend (the weights are softmax([Sa, Sb]))
+    sa = inp.lse_a[idx].to(torch.float64); sb = inp.lse_b[idx].to(torch.float64)
+    w = torch.softmax(torch.stack([sa, sb], -1), -1).nan_to_num(0.0)
+    va = torch.nan_to_num(inp.v_a[idx].to(torch.float64), nan=0.0, posinf=0.0, neginf=0.0)
+    vb = torch.nan_to_num(inp.v_b[idx].to(torch.float64), nan=0.0, posinf=0.0, neginf=0.0)
+    floor = 2.0 ** -22 * ((w[..., 0:1] * va).abs() + (w[..., 1:2] * vb).abs()).numpy()
+    stats = check_values(f64(v[idx]), ov, inp.dtype, extra=floor, what=f"merge {tuple(inp.v_a.shape)}")
+    if with_lse:
+        stats["max_lse_err"] = check_lse(s[idx].numpy(), os_, what=f"merge lse {tuple(inp.v_a.shape)}")
+    return stats
+
+
+def sample_rows(T, n=192, seed=0):
+    if T <= n:
+        return np.arange(T)
+    rng = np.random.default_rng(seed)
+    pick = rng.choice(T, size=n, replace=False)
+    return np.unique(np.concatenate([[0, 1, T - 2, T - 1], pick]))
+
+
+# ---------------------------------------------------------------------------------------------
+# the named configurations
+# ---------------------------------------------------------------------------------------------
+
+def test_config1_fused_add_rmsnorm():
+    stats = run_rmsnorm(wl.config1())
+    assert stats["max_err_ulp"] <= 2.0
+
+
+def test_config2_silu_and_mul():
+    stats = run_silu(wl.config2())
+    assert stats["max_err_ulp"] <= 2.0
+
+
+def test_config3_merge_attn_states_lse():
+    inp = wl.config3()
+    both = torch.isinf(inp.lse_a) & torch.isinf(inp.lse_b)
+    one = torch.isinf(inp.lse_a) ^ torch.isinf(inp.lse_b)
+    assert both.sum() >= 4 and one.sum() > 50
+    run_merge(inp)
+
+
+@pytest.mark.parametrize("dtype", [BF16, FP16])
+@pytest.mark.parametrize("H", wl.SWEEP_H)
+@pytest.mark.parametrize("T", wl.SWEEP_T)
+def test_config4_rmsnorm_sweep(dtype, T, H):
+    inp = wl.config4_point(dtype, T, H)
+    run_rmsnorm(inp, rows=sample_rows(T))
+
+
+def test_config5_chain_shapes():
+    """Full-size chain shapes in the launch configuration the benchmark times; sampled rows."""
+    cfg = wl.config5()
+    run_rmsnorm(cfg["rmsnorm"], rows=sample_rows(wl.CHAIN_T, seed=1))
+    run_silu(cfg["silu"], rows=sample_rows(wl.CHAIN_T, n=64, seed=2))
+    run_merge(cfg["merge"], tokens=sample_rows(wl.CHAIN_T, seed=3))
+
+
+# ---------------------------------------------------------------------------------------------
+# shapes: tiny, ragged, several tiles, odd alignment
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype", [BF16, FP16])
+@pytest.mark.parametrize("H", [1, 2, 3, 7, 8, 9, 33, 250, 1000, 4100, 4101, 4098, 8190, 11008, 14336,
+                               32768, 32776, 40000, 65538])
+def test_rmsnorm_widths(dtype, H):
+    T = 3 if H > 20000 else 5
+    run_rmsnorm(wl.rmsnorm_inputs(T, H, dtype, eps=1e-5, seed=H))
+
+
+@pytest.mark.parametrize("offset", [1, 2, 4, 8])
+@pytest.mark.parametrize("H", [4096, 4100, 520])
+def test_rmsnorm_pointer_offsets(offset, H):
+    run_rmsnorm(wl.rmsnorm_inputs(7, H, BF16, eps=1e-6, seed=offset), offset=offset)
+
+
+def test_rmsnorm_closed_forms_on_gpu():
+    # constant row -> sign(c) * w ; zero row -> 0
+    H = 4096
+    w = wl.rmsnorm_inputs(1, H, BF16, seed=5).weight
+    x = torch.full((3, H), 0.75, dtype=torch.bfloat16); r = torch.full((3, H), 1.25, dtype=torch.bfloat16)
+    x[1] = -2.0; r[1] = -1.0; x[2] = 1.5; r[2] = -1.5
+    gx, gr, gw = Guarded(x), Guarded(r), Guarded(w)
+    astra.astra_fused_add_rmsnorm(gx.t, gr.t, gw.t, 1e-6)
+    y = gx.host()
+    assert torch.equal(y[0], w) and torch.equal(y[1], -w) and bool((y[2] == 0).all())
+    assert bool((gr.host()[0] == 2.0).all()) and bool((gr.host()[2] == 0).all())
+
+
+def test_rmsnorm_on_side_stream_and_repeatable():
+    inp = wl.rmsnorm_inputs(300, 5120, BF16, eps=1e-5, seed=12)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        a = run_rmsnorm(inp, stream=s)
+    b = run_rmsnorm(inp)
+    assert a == b
+
+
+@pytest.mark.parametrize("dtype", [BF16, FP16])
+@pytest.mark.parametrize("D", [1, 2, 7, 8, 9, 100, 1000, 4096, 5120, 12288, 14336, 14340, 14342, 14337])
+def test_silu_widths(dtype, D):
+    run_silu(wl.silu_inputs(5, D, dtype, std=2.0, seed=D))
+
+
+@pytest.mark.parametrize("offset", [1, 2, 4])
+def test_silu_pointer_offsets(offset):
+    run_silu(wl.silu_inputs(9, 4096, BF16, seed=offset), offset=offset)
+
+
+def test_silu_extreme_gates():
+    vals = [0.0, -0.0, 1e-30, -1e-30, 20.0, -20.0, 87.0, -87.0, 88.5, -88.5, 100.0, -100.0, 1e4, -1e4,
+            3e38, -3e38, 0.5, -0.5]
+    a = torch.tensor(vals, dtype=torch.float32).repeat(8)
+    b = torch.linspace(-1, 1, a.numel())
+    row = torch.cat([a, b]).to(torch.bfloat16).reshape(1, -1)
+    run_silu(wl.SiluInputs(row, BF16))
+    row16 = torch.cat([a.clamp(-6e4, 6e4), b]).to(torch.float16).reshape(1, -1)
+    run_silu(wl.SiluInputs(row16, FP16))
+
+
+@pytest.mark.parametrize("dtype", [BF16, FP16])
+@pytest.mark.parametrize("Hh,D", [(1, 1), (3, 7), (3, 8), (2, 9), (32, 128), (40, 128), (32, 256), (5, 80),
+                                  (7, 64), (3, 130), (2, 1028), (1, 4100)])
+def test_merge_shapes(dtype, Hh, D):
+    run_merge(wl.merge_inputs(37, Hh, D, dtype, seed=Hh * 1000 + D, neg_inf_frac=0.05))
+
+
+@pytest.mark.parametrize("offset", [1, 2, 4])
+def test_merge_pointer_offsets(offset):
+    run_merge(wl.merge_inputs(33, 8, 128, BF16, seed=offset), offset=offset)
+
+
+@pytest.mark.parametrize("in_place", ["a", "b"])
+def test_merge_in_place_values(in_place):
+    run_merge(wl.merge_inputs(129, 32, 128, BF16, seed=9), in_place=in_place)
+
+
+def test_merge_without_lse_output():
+    run_merge(wl.merge_inputs(65, 4, 128, BF16, seed=10), with_lse=False)
+
+
+def test_merge_special_scores():
+    """Equal scores -> mean and +ln 2; one -inf -> the other state, bit for bit, even when the empty
+    side holds Inf/NaN; both -inf -> zeros and -inf; +inf / NaN scores -> NaN."""
+    T, Hh, D = 8, 1, 128
+    inp = wl.merge_inputs(T, Hh, D, BF16, seed=3, neg_inf_frac=0.0, forced_both_neg_inf=0)
+    ninf, inf, nan = float("-inf"), float("inf"), float("nan")
+    inp.lse_a[:, 0] = torch.tensor([1.5, 2.0, ninf, ninf, 3.0, inf, nan, -40.0])
+    inp.lse_b[:, 0] = torch.tensor([1.5, ninf, -7.0, ninf, ninf, 0.0, 0.0, -40.0])
+    inp.v_b[4, 0, :4] = torch.tensor([inf, -inf, nan, 1.0], dtype=torch.bfloat16)  # garbage on the empty side
+    inp.v_a[2, 0, :2] = torch.tensor([nan, inf], dtype=torch.bfloat16)
+    ga, gb = Guarded(inp.v_a), Guarded(inp.v_b)
+    gsa, gsb = Guarded(inp.lse_a), Guarded(inp.lse_b)
+    go, gso = Guarded(torch.zeros_like(inp.v_a)), Guarded(torch.zeros((T, Hh), dtype=torch.float32))
+    astra.astra_merge_attn_states_lse(go.t, gso.t, ga.t, gsa.t, gb.t, gsb.t)
+    v, s = go.host(), gso.host()
+    assert torch.equal(v[1], inp.v_a[1]) and s[1, 0] == 2.0
+    assert torch.equal(v[2], inp.v_b[2]) and s[2, 0] == -7.0
+    assert bool((v[3] == 0).all()) and s[3, 0] == ninf
+    assert torch.equal(v[4], inp.v_a[4]) and s[4, 0] == 3.0
+    assert bool(v[5].isnan().all()) and bool(s[5].isnan().all())
+    assert bool(v[6].isnan().all()) and bool(s[6].isnan().all())
+    run_merge(inp)  # and the whole thing against the oracle
+
+
+# ---------------------------------------------------------------------------------------------
+# degenerate sizes and error codes through the C ABI
+# ---------------------------------------------------------------------------------------------
+
+def test_empty_inputs_launch_nothing():
+    lib = astra.load_library()
+    buf = torch.zeros(64, dtype=torch.bfloat16, device="cuda")
+    p = buf.data_ptr()
+    assert lib.astra_fused_add_rmsnorm(p, p + 32, p + 64, 0, 16, 1e-6, 0, None) == 0
+    assert lib.astra_silu_and_mul(p, p + 32, 0, 8, 0, None) == 0
+    assert lib.astra_merge_attn_states_lse(p, None, p, p, p, p, 0, 1, 8, 0, None) == 0
+    torch.cuda.synchronize()
+    assert bool((buf == 0).all())
+
+
+def test_binding_rejects_wrong_arguments():
+    x = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(TypeError):
+        astra.astra_fused_add_rmsnorm(x.cpu(), x, x[0], 1e-6)
+    with pytest.raises(ValueError):
+        astra.astra_fused_add_rmsnorm(x, x[:, :32], x[0], 1e-6)
+    with pytest.raises(TypeError):
+        astra.astra_silu_and_mul(x[:, :32].contiguous().float(), x)
+    with pytest.raises(astra.AstraError) as e:
+        astra.astra_fused_add_rmsnorm(x, x, x[0].clone(), 1e-6)
+    assert e.value.status == 6
