@@ -1,0 +1,421 @@
+#!/usr/bin/env python
+"""Benchmark of the three memory-bound kernels on the Llama-3-8B prefill-shaped chain.
+
+One step = fused_add_rmsnorm [T,4096] -> silu_and_mul [T,2*14336] -> merge_attn_states_lse
+[T,32,128] at T = 8192, bf16, issued back to back on one stream (a timing sequence; no data flows
+between the three).  The metric is achieved HBM bandwidth: algorithmic (minimum) bytes of the step
+divided by device time, with per-kernel microseconds and GB/s measured by CUDA events inside the
+same timed region, and the roofline fraction against the measured copy bandwidth of the GPU.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl astra|reference] [--no-sweep]
+
+N > 1 (under torchrun): every rank runs its own T = 8192 batch (weak scaling; the operations are
+independent per row, so there is no collective on the data path); time is the max over ranks.
+`--impl reference` times the fp64 CPU oracle on the host cores instead (rank 0 only).
+Exactly one JSON line is printed on stdout by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2509_07506_b200 import workloads as wl  # noqa: E402
+
+METRIC = "achieved_hbm_bandwidth_llama3_8b_prefill_chain"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 7700.0
+FALLBACK_HBM_GBS = 6650.0
+L2_BYTES = 126 * 1024 * 1024
+
+# Per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
+# the ncu capture summarised under profiles/; None until a capture of the current kernel exists.
+DOMINANT_KERNEL_TRAFFIC_BYTES = None
+
+
+def chain_bytes(T: int) -> dict:
+    return {
+        "fused_add_rmsnorm": wl.rmsnorm_bytes(T, wl.CHAIN_H),
+        "silu_and_mul": wl.silu_bytes(T, wl.CHAIN_D),
+        "merge_attn_states_lse": wl.merge_bytes(T, wl.CHAIN_HEADS, wl.CHAIN_HEAD_DIM),
+    }
+
+
+def measured_peak() -> tuple[float, str]:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, device copy)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier copy measurement on this pool)"
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks: nvidia-smi sampled in a child process while the timed regions run (read-only queries)
+# ---------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.lines = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "25"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, windows) -> dict:
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, line in self.lines:
+            if not any(a <= ts <= b for a, b in windows):
+                continue
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {
+            "sm_mhz": statistics.median(sm) if sm else None,
+            "sm_max_mhz": max(smax) if smax else None,
+            "reasons": sorted(reasons),
+            "samples": len(sm),
+        }
+
+
+# ---------------------------------------------------------------------------------------------
+# the CUDA arm
+# ---------------------------------------------------------------------------------------------
+def device_chain(T: int, seed_offset: int, dev):
+    """Host (pinned) and device copies of one rank's chain inputs and outputs."""
+    cfg = wl.config5(T) if seed_offset == 0 else _config5_seeded(T, 4 + 1000 * seed_offset)
+    rms, silu, merge = cfg["rmsnorm"], cfg["silu"], cfg["merge"]
+    host_in = {
+        "x": rms.x, "residual": rms.residual, "weight": rms.weight, "silu_in": silu.input,
+        "v_a": merge.v_a, "v_b": merge.v_b, "lse_a": merge.lse_a, "lse_b": merge.lse_b,
+    }
+    host_in = {k: v.pin_memory() for k, v in host_in.items()}
+    d = {k: v.to(dev) for k, v in host_in.items()}
+    d["silu_out"] = torch.empty((T, wl.CHAIN_D), dtype=torch.bfloat16, device=dev)
+    d["v_out"] = torch.empty_like(d["v_a"])
+    d["lse_out"] = torch.empty_like(d["lse_a"])
+    host_out = {k: torch.empty(d[k].shape, dtype=d[k].dtype).pin_memory()
+                for k in ("x", "residual", "silu_out", "v_out", "lse_out")}
+    return cfg, host_in, d, host_out
+
+
+def _config5_seeded(T, seed):
+    g = torch.Generator(device="cpu"); g.manual_seed(seed)
+    return {"rmsnorm": wl.rmsnorm_inputs(T, wl.CHAIN_H, wl.BF16, eps=1e-5, g=g),
+            "silu": wl.silu_inputs(T, wl.CHAIN_D, wl.BF16, std=1.0, g=g),
+            "merge": wl.merge_inputs(T, wl.CHAIN_HEADS, wl.CHAIN_HEAD_DIM, wl.BF16, -10.0, 20.0, 0.0, 0, g=g)}
+
+
+def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
+    import paper_2509_07506_b200 as astra
+    import torch.distributed as dist
+
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    astra.load_library()  # fails loudly if the CUDA library is missing
+    T = args.tokens
+    eps = 1e-5
+    cfg, host_in, d, host_out = device_chain(T, rank, dev)
+    nbytes = chain_bytes(T)
+    step_bytes = sum(nbytes.values())
+
+    def step():
+        astra.astra_fused_add_rmsnorm(d["x"], d["residual"], d["weight"], eps)
+        astra.astra_silu_and_mul(d["silu_out"], d["silu_in"])
+        astra.astra_merge_attn_states_lse(d["v_out"], d["lse_out"], d["v_a"], d["lse_a"], d["v_b"], d["lse_b"])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    K, W = args.steps, args.warmup
+    for _ in range(W):
+        step()
+    barrier()
+
+    # ---- device-resident timed region: K steps, events around every kernel ----------------------
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    barrier()
+    t_wall0 = time.time()
+    for i in range(K):
+        ev[i][0].record()
+        astra.astra_fused_add_rmsnorm(d["x"], d["residual"], d["weight"], eps)
+        ev[i][1].record()
+        astra.astra_silu_and_mul(d["silu_out"], d["silu_in"])
+        ev[i][2].record()
+        astra.astra_merge_attn_states_lse(d["v_out"], d["lse_out"], d["v_a"], d["lse_a"], d["v_b"], d["lse_b"])
+        ev[i][3].record()
+    barrier()
+    t_wall1 = time.time()
+    total_ms = ev[0][0].elapsed_time(ev[K - 1][3])
+    names = ["fused_add_rmsnorm", "silu_and_mul", "merge_attn_states_lse"]
+    kernel_ms = {n: sum(ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(K)) / K for j, n in enumerate(names)}
+
+    # ---- end-to-end: pinned host -> device, three calls, device -> pinned host, every step --------
+    Ke = max(1, min(K, args.e2e_steps))
+    h2d = sum(v.numel() * v.element_size() for v in host_in.values())
+    d2h = sum(v.numel() * v.element_size() for v in host_out.values())
+
+    def e2e_step():
+        for k, v in host_in.items():
+            d[k].copy_(v, non_blocking=True)
+        step()
+        for k, v in host_out.items():
+            v.copy_(d[k], non_blocking=True)
+
+    for _ in range(min(2, W)):
+        e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall2 = time.time()
+    e0.record()
+    for _ in range(Ke):
+        e2e_step()
+    e1.record()
+    barrier()
+    t_wall3 = time.time()
+    e2e_ms = e0.elapsed_time(e1)
+
+    # ---- max over ranks -------------------------------------------------------------------------
+    times = torch.tensor([total_ms, e2e_ms] + [kernel_ms[n] for n in names], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(times[0]), float(times[1])
+    kernel_ms = {n: float(times[2 + j]) for j, n in enumerate(names)}
+
+    if sampler is not None:
+        sampler.stop()
+    if rank != 0:
+        return None
+
+    peak, peak_source = measured_peak()
+    value = world * step_bytes * K / (total_ms * 1e-3) / 1e9
+    per_kernel = {}
+    for n in names:
+        gbs = nbytes[n] / (kernel_ms[n] * 1e-3) / 1e9
+        per_kernel[n] = {"us_per_call": round(kernel_ms[n] * 1e3, 2), "algorithmic_bytes": nbytes[n],
+                         "gbs": round(gbs, 1), "frac_of_measured_peak": round(gbs / peak, 4),
+                         "frac_of_nominal_7700": round(gbs / NOMINAL_HBM_GBS, 4)}
+    dominant = max(names, key=lambda n: kernel_ms[n])
+    dom_gbs = nbytes[dominant] / (kernel_ms[dominant] * 1e-3) / 1e9
+    result = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": round(total_ms / K, 5), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32 arithmetic on bf16 storage", "data": "synthetic",
+        "config": {
+            "workload": f"configs[4]: Llama-3-8B prefill-shaped chain, T={T} per GPU, bf16: "
+                        f"fused_add_rmsnorm [{T},4096] -> silu_and_mul [{T},2*14336] -> "
+                        f"merge_attn_states_lse [{T},32,128]",
+            "tokens_per_gpu": T, "seed": 4,
+            "l2_policy": "inputs larger than L2: each step touches %.0f MB (L2 is 126 MB) and every kernel's "
+                         "own working set exceeds L2, so nothing is re-used across launches" % (step_bytes / 1e6),
+            "parallelism": "rows sharded across GPUs, no collective" if world > 1 else "single GPU",
+        },
+        "per_kernel": per_kernel,
+        "roofline": {"bound": "hbm", "kernel": dominant, "achieved": round(dom_gbs, 1), "peak": peak,
+                     "unit": "GB/s", "frac": round(dom_gbs / peak, 4), "traffic": DOMINANT_KERNEL_TRAFFIC_BYTES,
+                     "peak_source": peak_source, "algorithmic_bytes_per_launch": nbytes[dominant]},
+        "e2e": {"value": round(world * step_bytes * Ke / (e2e_ms * 1e-3) / 1e9, 2), "unit": UNIT,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": Ke,
+                "ms_per_step": round(e2e_ms / Ke, 3)},
+        "gpu_launches": 3 * K,
+        "clocks": sampler.summary([(t_wall0, t_wall1), (t_wall2, t_wall3)]) if sampler else None,
+    }
+    if world == 1 and not args.no_sweep:
+        result["large_shapes"] = large_shape_sweep(astra, dev, peak)
+    if world == 1 and not args.no_cpu:
+        result["cpu_baseline"] = oracle_baseline(cfg, rows=min(args.cpu_rows, T))
+    return result
+
+
+def _time_launches(fn, reps=100, warmup=20):
+    """Paper protocol: 20 warm-up launches, 100 timed, back to back; median of 5 batches (us/call)."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    out = []
+    for _ in range(5):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        out.append(a.elapsed_time(b) * 1e3 / reps)
+    return statistics.median(out)
+
+
+def large_shape_sweep(astra, dev, peak) -> list:
+    """The large-token points of the fused_add_rmsnorm sweep (T = 16384; both dtypes).  Each point's
+    working set (>= 268 MB) exceeds L2, so repeated launches on one buffer set stay HBM-bound."""
+    rows = []
+    T = 16384
+    for dtype, td in ((wl.BF16, torch.bfloat16), (wl.FP16, torch.float16)):
+        for H in wl.SWEEP_H:
+            x = torch.randn((T, H), device=dev, dtype=torch.float32).to(td)
+            r = torch.randn((T, H), device=dev, dtype=torch.float32).to(td)
+            w = torch.ones((H,), device=dev, dtype=td)
+            us = _time_launches(lambda: astra.astra_fused_add_rmsnorm(x, r, w, 1e-5))
+            b = wl.rmsnorm_bytes(T, H)
+            gbs = b / (us * 1e-6) / 1e9
+            rows.append({"kernel": "fused_add_rmsnorm", "dtype": wl.DTYPE_NAME[dtype], "T": T, "H": H,
+                         "us_per_call": round(us, 2), "gbs": round(gbs, 1), "frac_of_measured_peak": round(gbs / peak, 4)})
+            del x, r, w
+    return rows
+
+
+# ---------------------------------------------------------------------------------------------
+# the CPU arm: the oracle, as it stands, on the host cores
+# ---------------------------------------------------------------------------------------------
+def _oracle_pass(cfg, rows: int, nthreads: int) -> float:
+    """One pass of the three oracle functions over the first `rows` rows/tokens; seconds."""
+    import oracle
+    rms, silu, merge = cfg["rmsnorm"], cfg["silu"], cfg["merge"]
+    xb, rb, wb = wl.bits(rms.x[:rows]), wl.bits(rms.residual[:rows]), wl.bits(rms.weight)
+    sb = wl.bits(silu.input[:rows])
+    va, vb = wl.bits(merge.v_a[:rows]), wl.bits(merge.v_b[:rows])
+    la, lb = merge.lse_a[:rows].numpy(), merge.lse_b[:rows].numpy()
+    t0 = time.perf_counter()
+    oracle.fused_add_rmsnorm(xb, rb, wb, rms.eps, rms.dtype, nthreads=nthreads)
+    oracle.silu_and_mul(sb, silu.dtype, nthreads=nthreads)
+    oracle.merge_attn_states_lse(va, la, vb, lb, merge.dtype, nthreads=nthreads)
+    return time.perf_counter() - t0
+
+
+def oracle_baseline(cfg, rows: int) -> dict:
+    import oracle
+    oracle.build()
+    cores = len(os.sched_getaffinity(0))
+    _oracle_pass(cfg, min(rows, 64), cores)  # load the library, touch the pages
+    sec = min(_oracle_pass(cfg, rows, cores) for _ in range(2))
+    b = sum(chain_bytes(rows).values())
+    return {"value": round(b / sec / 1e9, 3), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {rows} rows/tokens of each of the three chain calls, best of 2 passes, "
+                      f"{sec:.2f} s per pass, OpenMP over rows on all {cores} host cores",
+            "seconds": round(sec, 3)}
+
+
+def run_reference(args, rank: int) -> dict | None:
+    if rank != 0:
+        return None
+    import oracle
+    oracle.build()
+    cores = len(os.sched_getaffinity(0))
+    probe_rows = 32
+    cfg = wl.config5(wl.CHAIN_T) if args.cpu_rows > 1024 else wl.config5(1024)
+    max_rows = cfg["rmsnorm"].x.shape[0]
+    _oracle_pass(cfg, probe_rows, cores)
+    t_probe = min(_oracle_pass(cfg, probe_rows, cores) for _ in range(3))
+    budget = 90.0  # seconds for the whole K + W run
+    rows = int(budget / max(1, args.steps + args.warmup) / (t_probe / probe_rows))
+    rows = max(1, min(rows, max_rows))
+    for _ in range(args.warmup):
+        _oracle_pass(cfg, rows, cores)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        _oracle_pass(cfg, rows, cores)
+    sec = time.perf_counter() - t0
+    b = sum(chain_bytes(rows).values())
+    value = round(b * args.steps / sec / 1e9, 3)
+    sample = (f"each step = the fp64 oracle over the first {rows} of 8192 rows/tokens of the three chain calls, "
+              f"OpenMP over rows on {cores} host cores")
+    return {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(sec / args.steps * 1e3, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "configs[4]: Llama-3-8B prefill-shaped chain (bounded sample of T=8192), bf16 storage",
+                   "sample": sample, "seed": 4},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+def main() -> int:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", choices=["astra", "reference"], default="astra")
+    ap.add_argument("--e2e-steps", type=int, default=10, help="steps of the host-to-host timed region")
+    ap.add_argument("--cpu-rows", type=int, default=8192, help="rows of the chain the CPU baseline covers")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the T=16384 fused_add_rmsnorm points")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU (oracle) baseline leg")
+    ap.add_argument("--tokens", type=int, default=wl.CHAIN_T,
+                    help="tokens per GPU; the benchmark's workload is the default (8192), smaller values "
+                         "are for profiler captures")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        res = run_reference(args, rank)
+        if res is not None:
+            print(json.dumps(res), flush=True)
+        return 0
+
+    if not torch.cuda.is_available():
+        print("bench.py: no CUDA device; the CUDA library has no CPU fallback", file=sys.stderr)
+        return 1
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    try:
+        res = run_astra(args, rank, world, local_rank)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+    if res is not None:
+        print(json.dumps(res), flush=True)
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

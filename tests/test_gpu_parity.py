@@ -103,7 +103,9 @@ def run_merge(inp: wl.MergeInputs, tokens=None, offset=0, in_place=None, with_ls
     torch.cuda.synchronize()
     for g in (ga, gb, gsa, gsb, go, gso):
         g.check()
-    assert torch.equal(gsa.host(), inp.lse_a) and torch.equal(gsb.host(), inp.lse_b)
+    # inputs untouched (bitwise: the scores may hold NaN)
+    assert torch.equal(gsa.host().view(torch.int32), inp.lse_a.view(torch.int32))
+    assert torch.equal(gsb.host().view(torch.int32), inp.lse_b.view(torch.int32))
     v, s = go.host(), gso.host()
     if not with_lse:
         assert bool((s == 123.0).all())
