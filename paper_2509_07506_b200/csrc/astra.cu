@@ -39,6 +39,26 @@ inline astra_status_t launch_status() {
     return cudaGetLastError() == cudaSuccess ? ASTRA_OK : ASTRA_ERR_CUDA;
 }
 
+// Every kernel is launched with programmatic stream serialization allowed: its blocks may be
+// scheduled while the previous kernel in the stream drains, and they wait (griddepcontrol.wait)
+// for that kernel to complete before their first global access.  Stream order is unchanged; the
+// launch latency and block prologue of back-to-back calls overlap the previous kernel's tail.
+template <typename... KArgs, typename... Args>
+inline void launch(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t stream,
+                   Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);  // failure is read back by launch_status()
+}
+
 constexpr int64_t kMaxVecsPerLaunch = (1ll << 31) - 1;  // flat vector indices are 31-bit
 
 // ---------------------------------------------------------------------------------------------
@@ -53,16 +73,18 @@ void launch_silu(uint16_t *out, const uint16_t *in, int64_t T, int64_t D, cudaSt
         const uint32_t total = static_cast<uint32_t>(rows * nvec);
         const uint32_t tile = THREADS * UNROLL;
         const uint32_t blocks = (total + tile - 1) / tile;
-        silu_and_mul_kernel<DT, VEC, UNROLL, THREADS><<<blocks, THREADS, 0, stream>>>(
-            out + t0 * D, in + t0 * 2 * D, total, FastDiv::make(static_cast<uint32_t>(nvec)), D);
+        launch(silu_and_mul_kernel<DT, VEC, UNROLL, THREADS>, blocks, THREADS, stream,
+               out + t0 * D, in + t0 * 2 * D, total, FastDiv::make(static_cast<uint32_t>(nvec)), D);
     }
 }
 
 template <int DT>
 void dispatch_silu(uint16_t *out, const uint16_t *in, int64_t T, int64_t D, cudaStream_t stream) {
     // each row is [a | b]: a starts at 2*D*t and b at 2*D*t + D, so D itself must be a multiple of VEC
+    // One 16-byte vector per thread and 256-thread blocks: the smallest work quantum that still
+    // keeps the block scheduler ahead, which gives the shortest drain at the end of the grid.
     switch (pick_vec(8, D, out, in)) {
-        case 8: launch_silu<DT, 8, 2, 256>(out, in, T, D, stream); break;
+        case 8: launch_silu<DT, 8, 1, 256>(out, in, T, D, stream); break;
         case 4: launch_silu<DT, 4, 4, 256>(out, in, T, D, stream); break;
         case 2: launch_silu<DT, 2, 4, 256>(out, in, T, D, stream); break;
         default: launch_silu<DT, 1, 4, 256>(out, in, T, D, stream); break;
@@ -83,9 +105,9 @@ void launch_merge(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const fl
         const uint32_t total = static_cast<uint32_t>(rows * nvec);
         const uint32_t tile = THREADS * UNROLL;
         const uint32_t blocks = (total + tile - 1) / tile;
-        merge_attn_states_lse_kernel<DT, VEC, UNROLL, THREADS><<<blocks, THREADS, 0, stream>>>(
-            v_out + r0 * D, lse_out ? lse_out + r0 : nullptr, v_a + r0 * D, lse_a + r0, v_b + r0 * D,
-            lse_b + r0, total, FastDiv::make(static_cast<uint32_t>(nvec)));
+        launch(merge_attn_states_lse_kernel<DT, VEC, UNROLL, THREADS>, blocks, THREADS, stream,
+               v_out + r0 * D, lse_out ? lse_out + r0 : nullptr, v_a + r0 * D, lse_a + r0, v_b + r0 * D,
+               lse_b + r0, total, FastDiv::make(static_cast<uint32_t>(nvec)));
     }
 }
 
@@ -93,7 +115,8 @@ template <int DT>
 void dispatch_merge(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
                     const uint16_t *v_b, const float *lse_b, int64_t rows, int64_t D,
                     cudaStream_t stream) {
-    switch (pick_vec(8, D, v_out, v_a, v_b)) {
+    switch (pick_vec(16, D, v_out, v_a, v_b)) {
+        case 16: launch_merge<DT, 16, 1, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream); break;
         case 8: launch_merge<DT, 8, 2, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream); break;
         case 4: launch_merge<DT, 4, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream); break;
         case 2: launch_merge<DT, 2, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream); break;
@@ -108,41 +131,46 @@ constexpr int kMaxGridX = 2147483647;
 
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
+template <int DT, int VEC, int VPT>
+inline void launch_rmsnorm_reg(unsigned rows, int threads, cudaStream_t stream, uint16_t *x, uint16_t *r,
+                               const uint16_t *w, int H, float eps, float inv_H) {
+    // at most 64 elements per thread are ever selected; wider combinations are not instantiated
+    if constexpr (VEC * VPT <= 64)
+        launch(fused_add_rmsnorm_reg_kernel<DT, VEC, VPT>, rows, threads, stream, x, r, w, H, eps, inv_H);
+}
+
+// Register-resident rows: VPT vectors per thread with blockDim = ceil(nvec / VPT) rounded up to a warp.
+// 16 elements per thread (32 bytes of x and of r in flight per thread) with 256..1024 threads
+// measured best; up to 64 elements per thread are used for wider rows, with the block size capped
+// so the row still fits the register file.  Rows wider than that take the two-sweep kernel.
 template <int DT, int VEC>
 void launch_rmsnorm(uint16_t *x, uint16_t *r, const uint16_t *w, int64_t T, int H, float eps,
                     cudaStream_t stream) {
     const int nvec = H / VEC;
     const float inv_H = 1.0f / static_cast<float>(H);
-    // vectors per thread: aim for 32 elements (64 bytes of x and 64 of r in flight) per thread,
-    // within 128..1024 threads per row
-    constexpr int kTargetVpt = 32 / VEC < 1 ? 1 : 32 / VEC;
+    // start at 16 elements per thread; widen the per-thread share only if the row needs more
+    // threads than that share allows, narrow it if the block would fall under 128 threads
+    int vpt = 16 / VEC < 1 ? 1 : 16 / VEC;
+    auto threads_for = [&](int v) { return round_up((nvec + v - 1) / v, 32); };
+    while (vpt < 64 / VEC && threads_for(vpt) > rmsnorm_reg_max_threads(VEC, vpt)) vpt <<= 1;
+    while (vpt > 1 && threads_for(vpt) < 128) vpt >>= 1;
+    const int threads = threads_for(vpt);
+    const bool fits = threads <= rmsnorm_reg_max_threads(VEC, vpt);
     for (int64_t t0 = 0; t0 < T; t0 += kMaxGridX) {
-        const int rows = static_cast<int>(T - t0 < kMaxGridX ? T - t0 : kMaxGridX);
+        const unsigned rows = static_cast<unsigned>(T - t0 < kMaxGridX ? T - t0 : kMaxGridX);
         uint16_t *xs = x + t0 * H, *rs = r + t0 * H;
-        int vpt = kTargetVpt;
-        int threads = round_up((nvec + vpt - 1) / vpt, 32);
-        while (threads < 128 && vpt > 1) {
-            vpt >>= 1;
-            threads = round_up((nvec + vpt - 1) / vpt, 32);
+        if (!fits) {
+            launch(fused_add_rmsnorm_twopass_kernel<DT, VEC>, rows, 1024, stream, xs, rs, w, H, eps, inv_H);
+            continue;
         }
-        if (threads <= 1024 && kTargetVpt >= vpt) {
-#define ASTRA_RMS_CASE(V)                                                                        \
-    case V:                                                                                      \
-        if constexpr (V <= kTargetVpt)                                                           \
-            fused_add_rmsnorm_reg_kernel<DT, VEC, V><<<rows, threads, 0, stream>>>(xs, rs, w, H, eps, inv_H); \
-        break;
-            switch (vpt) {
-                ASTRA_RMS_CASE(1)
-                ASTRA_RMS_CASE(2)
-                ASTRA_RMS_CASE(4)
-                ASTRA_RMS_CASE(8)
-                ASTRA_RMS_CASE(16)
-                ASTRA_RMS_CASE(32)
-                default: break;
-            }
-#undef ASTRA_RMS_CASE
-        } else {
-            fused_add_rmsnorm_twopass_kernel<DT, VEC><<<rows, 1024, 0, stream>>>(xs, rs, w, H, eps, inv_H);
+        switch (vpt) {
+            case 1: launch_rmsnorm_reg<DT, VEC, 1>(rows, threads, stream, xs, rs, w, H, eps, inv_H); break;
+            case 2: launch_rmsnorm_reg<DT, VEC, 2>(rows, threads, stream, xs, rs, w, H, eps, inv_H); break;
+            case 4: launch_rmsnorm_reg<DT, VEC, 4>(rows, threads, stream, xs, rs, w, H, eps, inv_H); break;
+            case 8: launch_rmsnorm_reg<DT, VEC, 8>(rows, threads, stream, xs, rs, w, H, eps, inv_H); break;
+            case 16: launch_rmsnorm_reg<DT, VEC, 16>(rows, threads, stream, xs, rs, w, H, eps, inv_H); break;
+            case 32: launch_rmsnorm_reg<DT, VEC, 32>(rows, threads, stream, xs, rs, w, H, eps, inv_H); break;
+            default: launch_rmsnorm_reg<DT, VEC, 64>(rows, threads, stream, xs, rs, w, H, eps, inv_H); break;
         }
     }
 }

@@ -30,10 +30,17 @@ __device__ __forceinline__ float block_sum(float v, float *slots) {
     return t;
 }
 
+// Largest block the register-resident kernel may be launched with, by vectors per thread: the
+// row's binary32 sums (VPT * VEC registers) plus its packed inputs must fit the register file.
+__host__ __device__ constexpr int rmsnorm_reg_max_threads(int vec, int vpt) {
+    return vec * vpt <= 16 ? 1024 : (vec * vpt <= 32 ? 512 : 256);
+}
+
 // Register-resident row: thread i owns vectors i, i + blockDim.x, ... (at most VPT of them).
-// Requires nvec = H / VEC <= VPT * blockDim.x.
-template <int DT, int VEC, int VPT>
-__global__ void fused_add_rmsnorm_reg_kernel(uint16_t *x, uint16_t *residual,
+// Requires nvec = H / VEC <= VPT * blockDim.x and blockDim.x <= rmsnorm_reg_max_threads(VEC, VPT).
+template <int DT, int VEC, int VPT, Ld LDH = Ld::Stream, St STH = St::Stream>
+__global__ void __launch_bounds__(rmsnorm_reg_max_threads(VEC, VPT))
+fused_add_rmsnorm_reg_kernel(uint16_t *x, uint16_t *residual,
                                              const uint16_t *__restrict__ weight,
                                              int H, float eps, float inv_H) {
     __shared__ float slots[kMaxWarps];
@@ -41,6 +48,8 @@ __global__ void fused_add_rmsnorm_reg_kernel(uint16_t *x, uint16_t *residual,
     const int64_t row_off = static_cast<int64_t>(blockIdx.x) * H;
     uint16_t *xr = x + row_off;
     uint16_t *rr = residual + row_off;
+    grid_dependency_wait();
+    grid_launch_dependents();
 
     Pack<VEC> px[VPT], pr[VPT], pw[VPT];
 #pragma unroll
@@ -48,8 +57,8 @@ __global__ void fused_add_rmsnorm_reg_kernel(uint16_t *x, uint16_t *residual,
         const int v = threadIdx.x + i * blockDim.x;
         if (v < nvec) {
             // x and residual are rewritten by this same thread below: coherent loads, not .nc
-            px[i] = load<VEC, Ld::Stream>(xr + v * VEC);
-            pr[i] = load<VEC, Ld::Stream>(rr + v * VEC);
+            px[i] = load<VEC, LDH>(xr + v * VEC);
+            pr[i] = load<VEC, LDH>(rr + v * VEC);
         }
     }
 #pragma unroll
@@ -72,7 +81,7 @@ __global__ void fused_add_rmsnorm_reg_kernel(uint16_t *x, uint16_t *residual,
                 s[i][k] = fx[k] + fr[k];  // the one binary32 add
                 acc = fmaf(s[i][k], s[i][k], acc);
             }
-            store<VEC, St::Stream>(rr + v * VEC, narrow<DT, VEC>(s[i]));
+            store<VEC, STH>(rr + v * VEC, narrow<DT, VEC>(s[i]));
         }
     }
 
@@ -87,7 +96,7 @@ __global__ void fused_add_rmsnorm_reg_kernel(uint16_t *x, uint16_t *residual,
             widen<DT, VEC>(pw[i], fw);
 #pragma unroll
             for (int k = 0; k < VEC; ++k) fy[k] = s[i][k] * rstd * fw[k];
-            store<VEC, St::Stream>(xr + v * VEC, narrow<DT, VEC>(fy));
+            store<VEC, STH>(xr + v * VEC, narrow<DT, VEC>(fy));
         }
     }
 }
@@ -105,6 +114,8 @@ __global__ void fused_add_rmsnorm_twopass_kernel(uint16_t *x, uint16_t *residual
     const int64_t row_off = static_cast<int64_t>(blockIdx.x) * H;
     uint16_t *xr = x + row_off;
     uint16_t *rr = residual + row_off;
+    grid_dependency_wait();
+    grid_launch_dependents();
 
     float acc = 0.f;
     for (int v = threadIdx.x; v < nvec; v += blockDim.x) {

@@ -37,7 +37,10 @@ __device__ __forceinline__ MergeWeights merge_weights(float sa, float sb) {
     const bool a_is_hi = sa >= sb;
     r.wa = a_is_hi ? w_hi : w_lo;
     r.wb = a_is_hi ? w_lo : w_hi;
-    r.lse = m + log1pf(t);
+    // log(1 + t) with 1 + t in [1, 2]: lg2.approx is within about 2^-22 absolute there
+    float l2;
+    asm("lg2.approx.f32 %0, %1;" : "=f"(l2) : "f"(1.0f + t));
+    r.lse = fmaf(l2, 0.6931471805599453f, m);
     // +inf or NaN scores are outside the domain (e^{S} / e^{S} = inf / inf): everything becomes NaN.
     if (!(m < INFINITY) || sa != sa || sb != sb) { r.wa = r.wb = r.lse = __int_as_float(0x7fc00000); }
     r.use_a = !(r.wa == 0.f);
@@ -46,13 +49,15 @@ __device__ __forceinline__ MergeWeights merge_weights(float sa, float sb) {
 }
 
 // Flat indexing over vectors of VEC elements: vector v belongs to row = v / nvec (row = token*Hh+head).
-template <int DT, int VEC, int UNROLL, int THREADS>
+template <int DT, int VEC, int UNROLL, int THREADS, Ld LDH = Ld::Stream, St STH = St::Stream>
 __global__ void __launch_bounds__(THREADS)
 merge_attn_states_lse_kernel(uint16_t *v_out, float *lse_out,
                              const uint16_t *v_a, const float *lse_a,
                              const uint16_t *v_b, const float *lse_b,
                              uint32_t total_vecs, FastDiv nvec) {
     const uint32_t base = blockIdx.x * (THREADS * UNROLL) + threadIdx.x;
+    grid_dependency_wait();
+    grid_launch_dependents();
     Pack<VEC> a[UNROLL], b[UNROLL];
     float sa[UNROLL], sb[UNROLL];
     uint32_t row[UNROLL];
@@ -63,8 +68,8 @@ merge_attn_states_lse_kernel(uint16_t *v_out, float *lse_out,
             row[j] = nvec.div(v);
             // v_out may be exactly v_a or v_b, so these are ordinary (coherent) loads; the thread
             // that reads a vector is the only one that writes it
-            a[j] = load<VEC, Ld::Stream>(v_a + static_cast<int64_t>(v) * VEC);
-            b[j] = load<VEC, Ld::Stream>(v_b + static_cast<int64_t>(v) * VEC);
+            a[j] = load<VEC, LDH>(v_a + static_cast<int64_t>(v) * VEC);
+            b[j] = load<VEC, LDH>(v_b + static_cast<int64_t>(v) * VEC);
             sa[j] = lse_a[row[j]];
             sb[j] = lse_b[row[j]];
         }
@@ -83,7 +88,7 @@ merge_attn_states_lse_kernel(uint16_t *v_out, float *lse_out,
                 const float ta = mw.use_a ? fa[i] * mw.wa : 0.f;
                 fo[i] = mw.use_b ? fmaf(fb[i], mw.wb, ta) : ta;
             }
-            store<VEC, St::Stream>(v_out + static_cast<int64_t>(v) * VEC, narrow<DT, VEC>(fo));
+            store<VEC, STH>(v_out + static_cast<int64_t>(v) * VEC, narrow<DT, VEC>(fo));
             if (lse_out != nullptr && v == row[j] * nvec.d) lse_out[row[j]] = mw.lse;
         }
     }

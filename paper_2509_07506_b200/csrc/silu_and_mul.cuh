@@ -4,7 +4,9 @@
 // vectors of VEC elements; all its 2*UNROLL loads are issued before the first use so that enough
 // bytes are in flight per SM to cover HBM latency.  The sigmoid costs two special-function ops per
 // element (ex2 and rcp, the fast-math forms the paper's optimised kernel also turns to), in
-// binary32, with one rounding at the store.
+// binary32, with one rounding at the store.  Instruction count matters even though the kernel is
+// HBM-bound: under a sustained power cap the SM clock (and with it the on-chip fabric) drops as
+// issue activity rises, so the arithmetic is kept to the packed two-wide forms.
 #pragma once
 
 #include "vec.cuh"
@@ -12,24 +14,46 @@
 namespace astra {
 
 // SiLU(a) * b in binary32, in the overflow-free form: with t = e^{-|a|} in [0, 1],
-// sigmoid(a) = 1/(1+t) for a >= 0 and t/(1+t) for a < 0.  The reciprocal's argument stays in [1, 2].
-// ex2 is the non-flushing form so that e^{-|a|} below 2^-126 still yields the (tiny but
-// representable) product a * e^{a} * b instead of zero.
+// sigmoid(a) = 1/(1+t) for a >= 0 and t/(1+t) for a < 0, so the reciprocal's argument stays in
+// [1, 2].  t is formed as h*h with h = e^{-|a|/2} = 2^{-|a| * log2(e)/2}: h stays a normal number
+// down to |a| = 174, and the (non-flushing) product h*h reaches the subnormals, so a * e^{a} * b is
+// still produced where e^{a} alone is below 2^-126; beyond |a| = 174 the true result is below every
+// representable magnitude anyway.
+constexpr float kHalfLog2e = 0.7213475204444817f;
+
 __device__ __forceinline__ float silu_mul(float a, float b) {
-    float t, d;
-    asm("ex2.approx.f32 %0, %1;" : "=f"(t) : "f"(fabsf(a) * -1.4426950408889634f));
+    float h, d;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(h) : "f"(fabsf(a) * -kHalfLog2e));
+    const float t = h * h;
     asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(d) : "f"(1.0f + t));
-    const float sig = a >= 0.f ? d : t * d;
-    return a * sig * b;
+    return a * (d * (a >= 0.f ? 1.0f : t)) * b;
+}
+
+// Two elements at a time with the packed binary32 instructions of sm_100 (two multiplies or adds
+// per issue slot); the two special-function ops per element stay scalar.  Same arithmetic, element
+// by element, as silu_mul.
+__device__ __forceinline__ float2 silu_mul2(float2 a, float2 b) {
+    const float2 arg = __fmul2_rn(make_float2(fabsf(a.x), fabsf(a.y)), make_float2(-kHalfLog2e, -kHalfLog2e));
+    float2 h, d;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(h.x) : "f"(arg.x));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(h.y) : "f"(arg.y));
+    const float2 t = __fmul2_rn(h, h);
+    const float2 den = __fadd2_rn(t, make_float2(1.0f, 1.0f));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(d.x) : "f"(den.x));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(d.y) : "f"(den.y));
+    const float2 f = make_float2(a.x >= 0.f ? 1.0f : t.x, a.y >= 0.f ? 1.0f : t.y);
+    return __fmul2_rn(__fmul2_rn(a, __fmul2_rn(d, f)), b);
 }
 
 // Flat indexing: vector v of the output covers out[row, col*VEC .. col*VEC+VEC) with
 // row = v / nvec, col = v % nvec, nvec = D / VEC.  A block handles THREADS*UNROLL consecutive vectors.
-template <int DT, int VEC, int UNROLL, int THREADS>
+template <int DT, int VEC, int UNROLL, int THREADS, Ld LDH = Ld::StreamReadOnly, St STH = St::Stream>
 __global__ void __launch_bounds__(THREADS)
 silu_and_mul_kernel(uint16_t *__restrict__ out, const uint16_t *__restrict__ in,
                     uint32_t total_vecs, FastDiv nvec, int64_t D) {
     const uint32_t base = blockIdx.x * (THREADS * UNROLL) + threadIdx.x;
+    grid_dependency_wait();
+    grid_launch_dependents();
     Pack<VEC> a[UNROLL], b[UNROLL];
 #pragma unroll
     for (int j = 0; j < UNROLL; ++j) {
@@ -38,8 +62,8 @@ silu_and_mul_kernel(uint16_t *__restrict__ out, const uint16_t *__restrict__ in,
             const uint32_t row = nvec.div(v);
             const uint32_t col = v - row * nvec.d;
             const uint16_t *pa = in + (static_cast<int64_t>(row) * 2 * D + static_cast<int64_t>(col) * VEC);
-            a[j] = load<VEC, Ld::StreamReadOnly>(pa);
-            b[j] = load<VEC, Ld::StreamReadOnly>(pa + D);
+            a[j] = load<VEC, LDH>(pa);
+            b[j] = load<VEC, LDH>(pa + D);
         }
     }
 #pragma unroll
@@ -49,9 +73,17 @@ silu_and_mul_kernel(uint16_t *__restrict__ out, const uint16_t *__restrict__ in,
             float fa[VEC], fb[VEC], fo[VEC];
             widen<DT, VEC>(a[j], fa);
             widen<DT, VEC>(b[j], fb);
+            if constexpr (VEC == 1) {
+                fo[0] = silu_mul(fa[0], fb[0]);
+            } else {
 #pragma unroll
-            for (int i = 0; i < VEC; ++i) fo[i] = silu_mul(fa[i], fb[i]);
-            store<VEC, St::Stream>(out + static_cast<int64_t>(v) * VEC, narrow<DT, VEC>(fo));
+                for (int i = 0; i < VEC; i += 2) {
+                    const float2 o = silu_mul2(make_float2(fa[i], fa[i + 1]), make_float2(fb[i], fb[i + 1]));
+                    fo[i] = o.x;
+                    fo[i + 1] = o.y;
+                }
+            }
+            store<VEC, STH>(out + static_cast<int64_t>(v) * VEC, narrow<DT, VEC>(fo));
         }
     }
 }

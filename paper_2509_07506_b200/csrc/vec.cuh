@@ -182,6 +182,17 @@ template <int DT, int VEC> __device__ __forceinline__ Pack<VEC> narrow(const flo
 }
 
 // ---------------------------------------------------------------------------------------------
+// Programmatic dependent launch.  A kernel launched with the programmatic-stream-serialization
+// attribute may be scheduled while the previous kernel in the stream is still draining.  It must
+// not touch global memory before `grid_dependency_wait()` returns (the previous grid has then
+// completed and its writes are visible), so stream order is preserved; what overlaps is only the
+// launch latency and the block prologue.  `grid_launch_dependents()` lets the next kernel in the
+// stream do the same with respect to this one.  Both are no-ops for an ordinary launch.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// ---------------------------------------------------------------------------------------------
 // Division of a 31-bit index by a launch-constant divisor: q = (n * mul) >> shift, exact for
 // 0 <= n < 2^31 and 1 <= d < 2^31 with shift = 31 + ceil(log2 d), mul = ceil(2^shift / d) <= 2^32 - 1
 // (d = 1 is special-cased so that mul fits 32 bits).
