@@ -32,6 +32,7 @@ if ROOT not in sys.path:
 
 import torch  # noqa: E402
 
+from paper_2509_07506_b200 import multi  # noqa: E402
 from paper_2509_07506_b200 import workloads as wl  # noqa: E402
 
 METRIC = "achieved_hbm_bandwidth_llama3_8b_prefill_chain"
@@ -40,9 +41,14 @@ NOMINAL_HBM_GBS = 7700.0
 FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 * 1024 * 1024
 
-# Per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
-# the ncu capture summarised under profiles/; None until a capture of the current kernel exists.
-DOMINANT_KERNEL_TRAFFIC_BYTES = None
+# Per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) at T = 8192 from the ncu
+# capture summarised in profiles/chain_T8192_launch_list.md.  An entry is removed (reported as null)
+# whenever its kernel changes after the capture.
+NCU_TRAFFIC_BYTES_T8192 = {
+    "silu_and_mul": 670.2e6,
+    "fused_add_rmsnorm": 208.7e6,
+    "merge_attn_states_lse": 163.7e6,
+}
 
 
 def chain_bytes(T: int) -> dict:
@@ -239,9 +245,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
     e2e_ms = e0.elapsed_time(e1)
 
     # ---- max over ranks -------------------------------------------------------------------------
-    times = torch.tensor([total_ms, e2e_ms] + [kernel_ms[n] for n in names], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    times = multi.max_over_ranks([total_ms, e2e_ms] + [kernel_ms[n] for n in names], device=dev)
     total_ms, e2e_ms = float(times[0]), float(times[1])
     kernel_ms = {n: float(times[2 + j]) for j, n in enumerate(names)}
 
@@ -251,7 +255,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
         return None
 
     peak, peak_source = measured_peak()
-    value = world * step_bytes * K / (total_ms * 1e-3) / 1e9
+    value = multi.aggregate_rate(step_bytes, world, K, total_ms) / 1e9
     per_kernel = {}
     for n in names:
         gbs = nbytes[n] / (kernel_ms[n] * 1e-3) / 1e9
@@ -276,7 +280,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
         "per_kernel": per_kernel,
         "per_kernel_how": f"each kernel alone: {K} back-to-back launches between two CUDA events, after the chain region",
         "roofline": {"bound": "hbm", "kernel": dominant, "achieved": round(dom_gbs, 1), "peak": peak,
-                     "unit": "GB/s", "frac": round(dom_gbs / peak, 4), "traffic": DOMINANT_KERNEL_TRAFFIC_BYTES,
+                     "unit": "GB/s", "frac": round(dom_gbs / peak, 4), "traffic": NCU_TRAFFIC_BYTES_T8192.get(dominant) if T == wl.CHAIN_T else None,
                      "peak_source": peak_source, "algorithmic_bytes_per_launch": nbytes[dominant]},
         "e2e": {"value": round(world * step_bytes * Ke / (e2e_ms * 1e-3) / 1e9, 2), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": Ke,
@@ -366,7 +370,7 @@ def run_reference(args, rank: int) -> dict | None:
     cores = len(os.sched_getaffinity(0))
     probe_rows = 32
     cfg = wl.config5(wl.CHAIN_T) if args.cpu_rows > 1024 else wl.config5(1024)
-    max_rows = cfg["rmsnorm"].x.shape[0]
+    max_rows = min(cfg["rmsnorm"].x.shape[0], args.cpu_rows)
     _oracle_pass(cfg, probe_rows, cores)
     t_probe = min(_oracle_pass(cfg, probe_rows, cores) for _ in range(3))
     budget = 90.0  # seconds for the whole K + W run
@@ -412,9 +416,7 @@ def main() -> int:
     if args.warmup < 3:
         args.warmup = 3
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local_rank = multi.env_rank_world()
 
     if args.impl == "reference":
         res = run_reference(args, rank)
@@ -426,9 +428,7 @@ def main() -> int:
         print("bench.py: no CUDA device; the CUDA library has no CPU fallback", file=sys.stderr)
         return 1
     if world > 1:
-        import torch.distributed as dist
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        multi.init_process_group("nccl", torch.device("cuda", local_rank))
     try:
         res = run_astra(args, rank, world, local_rank)
     finally:
