@@ -289,7 +289,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
         "clocks": sampler.summary([(t_wall0, t_wall1), (t_wall2, t_wall3)]) if sampler else None,
     }
     if world == 1 and not args.no_sweep:
-        result["large_shapes"] = large_shape_sweep(astra, dev, peak)
+        result["shape_sweep"] = shape_sweep(astra, dev, peak)
     if world == 1 and not args.no_cpu:
         result["cpu_baseline"] = oracle_baseline(cfg, rows=min(args.cpu_rows, T))
     return result
@@ -312,22 +312,94 @@ def _time_launches(fn, reps=100, warmup=20):
     return statistics.median(out)
 
 
-def large_shape_sweep(astra, dev, peak) -> list:
-    """The large-token points of the fused_add_rmsnorm sweep (T = 16384; both dtypes).  Each point's
-    working set (>= 268 MB) exceeds L2, so repeated launches on one buffer set stay HBM-bound."""
+def _rotating(make, nbytes: int):
+    """Enough independent buffer sets that a pass over all of them exceeds twice the L2 size."""
+    n = max(1, min(64, -(-2 * L2_BYTES // max(1, nbytes))))
+    return [make() for _ in range(n)]
+
+
+def _time_sets(call, sets):
+    """us/call, cycling through the buffer sets (one set: L2-hot; several: every launch misses L2)."""
+    state = {"i": 0}
+
+    def fn():
+        call(sets[state["i"] % len(sets)])
+        state["i"] += 1
+    return _time_launches(fn)
+
+
+def _time_graph(call, sets, launches=100):
+    """us/call on the device alone: `launches` calls captured into one CUDA graph (cycling through the
+    buffer sets), replayed; removes the host's per-call cost, which dominates the small shapes."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for i in range(3):
+            call(sets[i % len(sets)])
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(launches):
+                call(sets[i % len(sets)])
+        out = []
+        for _ in range(7):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(side)
+            graph.replay()
+            b.record(side)
+            side.synchronize()
+            out.append(a.elapsed_time(b) * 1e3 / launches)
+    torch.cuda.current_stream().wait_stream(side)
+    return statistics.median(out[2:])
+
+
+def shape_sweep(astra, dev, peak) -> list:
+    """us/call for configs[0..2] and every point of the fused_add_rmsnorm sweep (configs[3]).
+    `us_hot` repeats one buffer set (it stays in L2 when it fits); `us_cold` cycles through enough
+    sets to defeat L2; `*_graph` are the same launches replayed from a CUDA graph (device time only).  Shapes whose working set exceeds L2 give the same number both ways and carry
+    the roofline fraction; the small ones are launch-latency bound and are reported in us only."""
     rows = []
-    T = 16384
-    for dtype, td in ((wl.BF16, torch.bfloat16), (wl.FP16, torch.float16)):
-        for H in wl.SWEEP_H:
-            x = torch.randn((T, H), device=dev, dtype=torch.float32).to(td)
-            r = torch.randn((T, H), device=dev, dtype=torch.float32).to(td)
-            w = torch.ones((H,), device=dev, dtype=td)
-            us = _time_launches(lambda: astra.astra_fused_add_rmsnorm(x, r, w, 1e-5))
-            b = wl.rmsnorm_bytes(T, H)
-            gbs = b / (us * 1e-6) / 1e9
-            rows.append({"kernel": "fused_add_rmsnorm", "dtype": wl.DTYPE_NAME[dtype], "T": T, "H": H,
-                         "us_per_call": round(us, 2), "gbs": round(gbs, 1), "frac_of_measured_peak": round(gbs / peak, 4)})
-            del x, r, w
+
+    def add(kernel, dtype, shape, nbytes, make, call):
+        one = [make()]
+        big = nbytes > 2 * L2_BYTES
+        many = one if big else _rotating(make, nbytes)
+        hot = _time_sets(call, one)
+        cold = hot if big else _time_sets(call, many)
+        row = {"kernel": kernel, "dtype": wl.DTYPE_NAME[dtype], "shape": shape, "algorithmic_bytes": nbytes,
+               "us_hot": round(hot, 2), "us_cold": round(cold, 2)}
+        if not big:  # device time without the host's launch cost
+            row["us_hot_graph"] = round(_time_graph(call, one), 2)
+            row["us_cold_graph"] = round(_time_graph(call, many), 2)
+        best = cold if big else row["us_cold_graph"]
+        gbs = nbytes / (best * 1e-6) / 1e9
+        row["gbs_cold"] = round(gbs, 1)
+        row["frac_of_measured_peak"] = round(gbs / peak, 4) if big else None
+        rows.append(row)
+
+    def rms(dtype, T, H):
+        td = wl.torch_dtype(dtype)
+        make = lambda: (torch.randn((T, H), device=dev).to(td), torch.randn((T, H), device=dev).to(td),  # noqa: E731
+                        torch.ones((H,), device=dev, dtype=td))
+        add("fused_add_rmsnorm", dtype, [T, H], wl.rmsnorm_bytes(T, H), make,
+            lambda b: astra.astra_fused_add_rmsnorm(b[0], b[1], b[2], 1e-5))
+
+    rms(wl.BF16, 16, 4096)                                            # configs[0]
+    T, D = 128, wl.CHAIN_D                                            # configs[1]
+    add("silu_and_mul", wl.BF16, [T, 2 * D], wl.silu_bytes(T, D),
+        lambda: (torch.empty((T, D), device=dev, dtype=torch.bfloat16),
+                 (2 * torch.randn((T, 2 * D), device=dev)).to(torch.bfloat16)),
+        lambda b: astra.astra_silu_and_mul(b[0], b[1]))
+    T, Hh, Dh = 512, 32, 128                                          # configs[2]
+    add("merge_attn_states_lse", wl.BF16, [T, Hh, Dh], wl.merge_bytes(T, Hh, Dh),
+        lambda: (torch.empty((T, Hh, Dh), device=dev, dtype=torch.bfloat16), torch.empty((T, Hh), device=dev),
+                 torch.randn((T, Hh, Dh), device=dev).to(torch.bfloat16), torch.rand((T, Hh), device=dev) * 20 - 5,
+                 torch.randn((T, Hh, Dh), device=dev).to(torch.bfloat16), torch.rand((T, Hh), device=dev) * 20 - 5),
+        lambda b: astra.astra_merge_attn_states_lse(b[0], b[1], b[2], b[3], b[4], b[5]))
+    for dtype in wl.SWEEP_DTYPES:                                     # configs[3]
+        for T in wl.SWEEP_T:
+            for H in wl.SWEEP_H:
+                rms(dtype, T, H)
     return rows
 
 
@@ -406,7 +478,7 @@ def main() -> int:
     ap.add_argument("--impl", choices=["astra", "reference"], default="astra")
     ap.add_argument("--e2e-steps", type=int, default=10, help="steps of the host-to-host timed region")
     ap.add_argument("--cpu-rows", type=int, default=8192, help="rows of the chain the CPU baseline covers")
-    ap.add_argument("--no-sweep", action="store_true", help="skip the T=16384 fused_add_rmsnorm points")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the per-shape timings of configs[0..3]")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU (oracle) baseline leg")
     ap.add_argument("--no-clocks", action="store_true", help="do not sample clocks with nvidia-smi")
     ap.add_argument("--tokens", type=int, default=wl.CHAIN_T,

@@ -95,6 +95,28 @@ def _stream(t: torch.Tensor, stream: Optional[torch.cuda.Stream]) -> int:
     return s.cuda_stream
 
 
+class _on_device:
+    """Make the tensor's device current for the duration of the call (the C side launches on the
+    current device); a no-op, and cheap, when it already is."""
+
+    __slots__ = ("idx", "prev")
+
+    def __init__(self, t: torch.Tensor):
+        self.idx = t.device.index
+        self.prev = None
+
+    def __enter__(self):
+        cur = torch.cuda.current_device()
+        if self.idx is not None and self.idx != cur:
+            self.prev = cur
+            torch.cuda.set_device(self.idx)
+
+    def __exit__(self, *exc):
+        if self.prev is not None:
+            torch.cuda.set_device(self.prev)
+        return False
+
+
 def astra_fused_add_rmsnorm(x: torch.Tensor, residual: torch.Tensor, weight: torch.Tensor,
                             eps: float, stream: Optional[torch.cuda.Stream] = None) -> None:
     """In place: residual <- x + residual, x <- RMSNorm(x + residual) * weight.  x, residual [T, H]."""
@@ -105,7 +127,7 @@ def astra_fused_add_rmsnorm(x: torch.Tensor, residual: torch.Tensor, weight: tor
     T, H = x.shape
     _check(residual, "residual", x.dtype, (T, H))
     _check(weight, "weight", x.dtype, (H,))
-    with torch.cuda.device(x.device):
+    with _on_device(x):
         st = load_library().astra_fused_add_rmsnorm(
             x.data_ptr(), residual.data_ptr(), weight.data_ptr(), T, H, float(eps), code,
             _stream(x, stream))
@@ -122,7 +144,7 @@ def astra_silu_and_mul(out: torch.Tensor, input: torch.Tensor,
         raise ValueError("input must be [T, 2*D]")
     T, D = input.shape[0], input.shape[1] // 2
     _check(out, "out", input.dtype, (T, D))
-    with torch.cuda.device(input.device):
+    with _on_device(input):
         st = load_library().astra_silu_and_mul(out.data_ptr(), input.data_ptr(), T, D, code,
                                                _stream(input, stream))
     if st != ASTRA_OK:
@@ -145,7 +167,7 @@ def astra_merge_attn_states_lse(v_out: torch.Tensor, lse_out: Optional[torch.Ten
     _check(lse_b, "lse_b", torch.float32, (T, Hh))
     if lse_out is not None:
         _check(lse_out, "lse_out", torch.float32, (T, Hh))
-    with torch.cuda.device(v_a.device):
+    with _on_device(v_a):
         st = load_library().astra_merge_attn_states_lse(
             v_out.data_ptr(), lse_out.data_ptr() if lse_out is not None else None,
             v_a.data_ptr(), lse_a.data_ptr(), v_b.data_ptr(), lse_b.data_ptr(),
