@@ -267,7 +267,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
     result = {
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": round(total_ms / K, 5), "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32 arithmetic on bf16 storage", "data": "synthetic",
+        "vs_baseline": None, "dtype": "f32", "storage_dtype": "bf16", "data": "synthetic",
         "config": {
             "workload": f"configs[4]: Llama-3-8B prefill-shaped chain, T={T} per GPU, bf16: "
                         f"fused_add_rmsnorm [{T},4096] -> silu_and_mul [{T},2*14336] -> "
@@ -290,6 +290,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
     }
     if world == 1 and not args.no_sweep:
         result["shape_sweep"] = shape_sweep(astra, dev, peak)
+        result["table4"] = table4_sweep(astra, dev, peak)
     if world == 1 and not args.no_cpu:
         result["cpu_baseline"] = oracle_baseline(cfg, rows=min(args.cpu_rows, T))
     return result
@@ -400,6 +401,41 @@ def shape_sweep(astra, dev, peak) -> list:
         for T in wl.SWEEP_T:
             for H in wl.SWEEP_H:
                 rms(dtype, T, H)
+    return rows
+
+
+def table4_sweep(astra, dev, peak) -> list:
+    """The paper's Table 4 shapes, fp16 (the type its fragments use): device us/call from a CUDA
+    graph, L2-hot and L2-cold, beside the paper's H100 figures (measured inside a serving framework
+    on another machine: context only)."""
+    rows = []
+    td = torch.float16
+    for kernel, shape, h100_base, h100_opt in wl.TABLE4:
+        if kernel == "merge_attn_states_lse":
+            T, Hh, Dh = shape
+            nbytes = wl.merge_bytes(T, Hh, Dh)
+            make = lambda: (torch.empty((T, Hh, Dh), device=dev, dtype=td), torch.empty((T, Hh), device=dev),  # noqa: E731
+                            torch.randn((T, Hh, Dh), device=dev).to(td), torch.rand((T, Hh), device=dev) * 20 - 5,
+                            torch.randn((T, Hh, Dh), device=dev).to(td), torch.rand((T, Hh), device=dev) * 20 - 5)
+            call = lambda b: astra.astra_merge_attn_states_lse(b[0], b[1], b[2], b[3], b[4], b[5])  # noqa: E731
+        elif kernel == "fused_add_rmsnorm":
+            T, H = shape
+            nbytes = wl.rmsnorm_bytes(T, H)
+            make = lambda: (torch.randn((T, H), device=dev).to(td), torch.randn((T, H), device=dev).to(td),  # noqa: E731
+                            torch.ones((H,), device=dev, dtype=td))
+            call = lambda b: astra.astra_fused_add_rmsnorm(b[0], b[1], b[2], 1e-6)  # noqa: E731
+        else:
+            T, D = shape
+            nbytes = wl.silu_bytes(T, D)
+            make = lambda: (torch.empty((T, D), device=dev, dtype=td), (2 * torch.randn((T, 2 * D), device=dev)).to(td))  # noqa: E731
+            call = lambda b: astra.astra_silu_and_mul(b[0], b[1])  # noqa: E731
+        one = [make()]
+        many = _rotating(make, nbytes)
+        rows.append({"kernel": kernel, "dtype": "fp16", "shape": list(shape), "algorithmic_bytes": nbytes,
+                     "us_eager": round(_time_sets(call, one), 2),
+                     "us_hot_graph": round(_time_graph(call, one), 2),
+                     "us_cold_graph": round(_time_graph(call, many), 2),
+                     "paper_h100_us_base": h100_base, "paper_h100_us_opt": h100_opt})
     return rows
 
 

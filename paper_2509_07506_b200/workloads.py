@@ -161,6 +161,38 @@ def config5(T: int = CHAIN_T) -> Dict[str, object]:
     return {"rmsnorm": rms, "silu": silu, "merge": merge}
 
 
+# ---- the twelve shapes of the paper's Table 4 (per-shape study) -----------------------------
+# (kernel, shape, paper's H100 time of its baseline kernel in us, of its optimised kernel in us).
+# The paper does not state the precision of these runs; its code fragments use 16-bit floats.
+# Shapes are [seq_len, heads, head_dim] for the merge and [batch, hidden] for the other two; for
+# silu_and_mul, hidden is read as the output width D (the input row is 2*D wide).
+TABLE4 = (
+    ("merge_attn_states_lse", (512, 32, 256), 32.9, 22.6),
+    ("merge_attn_states_lse", (512, 40, 128), 32.4, 20.6),
+    ("merge_attn_states_lse", (768, 32, 256), 32.5, 32.5),
+    ("merge_attn_states_lse", (512, 64, 128), 32.0, 28.2),
+    ("fused_add_rmsnorm", (256, 4096), 24.3, 18.3),
+    ("fused_add_rmsnorm", (1024, 4096), 34.0, 28.3),
+    ("fused_add_rmsnorm", (128, 11008), 25.0, 19.4),
+    ("fused_add_rmsnorm", (512, 14336), 46.1, 43.0),
+    ("silu_and_mul", (16, 4096), 20.9, 14.2),
+    ("silu_and_mul", (32, 5120), 20.3, 13.7),
+    ("silu_and_mul", (64, 8192), 20.3, 13.5),
+    ("silu_and_mul", (16, 12288), 20.4, 13.6),
+)
+
+
+def table4_inputs(kernel: str, shape, dtype: int = BF16, seed: int = 5):
+    """Seeded inputs for one Table 4 shape (same value distributions as configs[0..2])."""
+    if kernel == "merge_attn_states_lse":
+        return merge_inputs(shape[0], shape[1], shape[2], dtype, seed=seed)
+    if kernel == "fused_add_rmsnorm":
+        return rmsnorm_inputs(shape[0], shape[1], dtype, eps=1e-6, seed=seed)
+    if kernel == "silu_and_mul":
+        return silu_inputs(shape[0], shape[1], dtype, std=2.0, seed=seed)
+    raise ValueError(kernel)
+
+
 # ---- algorithmic (minimum) bytes per call -------------------------------------------------
 
 def rmsnorm_bytes(T: int, H: int, elem: int = 2) -> int:

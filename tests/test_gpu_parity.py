@@ -175,6 +175,14 @@ def test_config5_chain_shapes():
     run_merge(cfg["merge"], tokens=sample_rows(wl.CHAIN_T, seed=3))
 
 
+@pytest.mark.parametrize("dtype", [BF16, FP16])
+@pytest.mark.parametrize("kernel,shape", [(k, sh) for k, sh, _, _ in wl.TABLE4])
+def test_table4_shapes(dtype, kernel, shape):
+    """The twelve shapes of the paper's per-shape study (Table 4), all elements."""
+    inp = wl.table4_inputs(kernel, shape, dtype)
+    {"merge_attn_states_lse": run_merge, "fused_add_rmsnorm": run_rmsnorm, "silu_and_mul": run_silu}[kernel](inp)
+
+
 # ---------------------------------------------------------------------------------------------
 # shapes: tiny, ragged, several tiles, odd alignment
 # ---------------------------------------------------------------------------------------------
