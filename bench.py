@@ -291,6 +291,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
     if world == 1 and not args.no_sweep:
         result["shape_sweep"] = shape_sweep(astra, dev, peak)
         result["table4"] = table4_sweep(astra, dev, peak)
+        result["strided_variants"] = strided_variants(astra, dev, peak)
     if world == 1 and not args.no_cpu:
         result["cpu_baseline"] = oracle_baseline(cfg, rows=min(args.cpu_rows, T))
     return result
@@ -401,6 +402,42 @@ def shape_sweep(astra, dev, peak) -> list:
         for T in wl.SWEEP_T:
             for H in wl.SWEEP_H:
                 rms(dtype, T, H)
+    return rows
+
+
+def strided_variants(astra, dev, peak) -> list:
+    """The strided / out-of-place entry points at the chain shapes (T = 8192, bf16); each moves the
+    same algorithmic bytes as its plain counterpart, so the same roofline applies."""
+    T, H, D, Hh, Dh = wl.CHAIN_T, wl.CHAIN_H, wl.CHAIN_D, wl.CHAIN_HEADS, wl.CHAIN_HEAD_DIM
+    bf = torch.bfloat16
+    rows = []
+
+    def add(name, nbytes, fn):
+        us = _time_launches(fn)
+        gbs = nbytes / (us * 1e-6) / 1e9
+        rows.append({"call": name, "us_per_call": round(us, 2), "gbs": round(gbs, 1),
+                     "frac_of_measured_peak": round(gbs / peak, 4)})
+
+    x = torch.randn((T, H), device=dev).to(bf); r = torch.randn((T, H), device=dev).to(bf)
+    y = torch.empty_like(x); ro = torch.empty_like(x); w = torch.ones((H,), device=dev, dtype=bf)
+    add("astra_fused_add_rmsnorm_ex out-of-place [8192,4096]", wl.rmsnorm_bytes(T, H),
+        lambda: astra.astra_fused_add_rmsnorm_ex(y, ro, x, r, w, 1e-5))
+    wide = torch.randn((T, 2 * H + 256), device=dev).to(bf)
+    xs, rs = wide[:, :H], wide[:, H + 128:2 * H + 128]
+    add("astra_fused_add_rmsnorm_ex in place on slices of a [8192, 8448] buffer", wl.rmsnorm_bytes(T, H),
+        lambda: astra.astra_fused_add_rmsnorm_ex(xs, rs, xs, rs, w, 1e-5))
+    del x, r, y, ro, wide
+    gate = torch.randn((T, D), device=dev).to(bf); up = torch.randn((T, D), device=dev).to(bf)
+    out = torch.empty((T, D), device=dev, dtype=bf)
+    add("astra_silu_and_mul_ex separate gate and up tensors [8192,14336]", wl.silu_bytes(T, D),
+        lambda: astra.astra_silu_and_mul_ex(out, gate, up))
+    del gate, up, out
+    va = torch.randn((T, Hh, Dh), device=dev).to(bf); vb = torch.randn((T, Hh, Dh), device=dev).to(bf)
+    vo = torch.empty_like(va)
+    sa = (torch.rand((Hh, T), device=dev) * 30 - 10).t(); sb = (torch.rand((Hh, T), device=dev) * 30 - 10).t()
+    so = torch.empty((Hh, T), device=dev).t()
+    add("astra_merge_attn_states_lse_ex head-major scores [8192,32,128]", wl.merge_bytes(T, Hh, Dh),
+        lambda: astra.astra_merge_attn_states_lse_ex(vo, so, va, sa, vb, sb))
     return rows
 
 

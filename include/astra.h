@@ -95,6 +95,58 @@ astra_status_t astra_merge_attn_states_lse(void *v_out, float *lse_out,
                                            int64_t T, int64_t Hh, int64_t D,
                                            astra_dtype_t dtype, void *cuda_stream);
 
+/*
+ * Strided / out-of-place forms.  Same operations and arithmetic as above (Table 1); only the
+ * addressing differs.  All pitches and strides are in ELEMENTS and must be non-negative; the
+ * innermost dimension is always contiguous.  Rows of one tensor must not overlap each other
+ * (pitch >= row width), otherwise ASTRA_ERR_BAD_SHAPE.  Vector width is chosen from the width, the
+ * pitches and the base addresses, so slices of wider buffers work at any element alignment.
+ */
+
+/*
+ * fused_add_rmsnorm with separate outputs and row pitches.
+ *   y            [T, H] rows y_pitch apart             out: RMSNorm(x + residual) * weight
+ *   residual_out [T, H] rows residual_out_pitch apart  out: x + residual (one binary32 add, one rounding)
+ *   x, residual  [T, H] rows x_pitch / residual_pitch apart, in
+ * y may be exactly x (same address and pitch) and residual_out exactly residual; that is the
+ * in-place form, and astra_fused_add_rmsnorm(x, r, w, ...) is this call with y = x,
+ * residual_out = r and all pitches equal to H.  Any other overlap between an output and another
+ * operand gives ASTRA_ERR_OVERLAP.
+ */
+astra_status_t astra_fused_add_rmsnorm_ex(void *y, void *residual_out, const void *x,
+                                          const void *residual, const void *weight,
+                                          int64_t T, int64_t H,
+                                          int64_t y_pitch, int64_t residual_out_pitch,
+                                          int64_t x_pitch, int64_t residual_pitch,
+                                          float eps, astra_dtype_t dtype, void *cuda_stream);
+
+/*
+ * silu_and_mul with separately addressed gate and up operands.
+ *   gate [T, D] rows gate_pitch apart, up [T, D] rows up_pitch apart, out [T, D] rows out_pitch apart.
+ * The packed row [a | b] of astra_silu_and_mul is gate = input, up = input + D, both pitches 2*D.
+ * out must not overlap gate or up.
+ */
+astra_status_t astra_silu_and_mul_ex(void *out, const void *gate, const void *up,
+                                     int64_t T, int64_t D,
+                                     int64_t out_pitch, int64_t gate_pitch, int64_t up_pitch,
+                                     astra_dtype_t dtype, void *cuda_stream);
+
+/*
+ * merge_attn_states_lse for strided tensors.  `strides` is a HOST array of 12 element strides:
+ *   { v_a token, v_a head, v_b token, v_b head, v_out token, v_out head,
+ *     lse_a token, lse_a head, lse_b token, lse_b head, lse_out token, lse_out head }.
+ * head_dim is contiguous in the value tensors.  Scores stored head-major ([Hh, T]) are
+ * { token stride 1, head stride T }.  T * Hh must be below 2^31.  Aliasing rules as for
+ * astra_merge_attn_states_lse: v_out may be exactly v_a or v_b (same address and strides);
+ * lse_out may be NULL (its two strides are then ignored).
+ */
+astra_status_t astra_merge_attn_states_lse_ex(void *v_out, float *lse_out,
+                                              const void *v_a, const float *lse_a,
+                                              const void *v_b, const float *lse_b,
+                                              int64_t T, int64_t Hh, int64_t D,
+                                              const int64_t *strides,
+                                              astra_dtype_t dtype, void *cuda_stream);
+
 /* Static, NUL-terminated description of a status code (never NULL). */
 const char *astra_status_string(astra_status_t status);
 

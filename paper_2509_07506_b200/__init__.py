@@ -7,8 +7,11 @@ load the library; the first call does, and fails loudly if it has not been built
 from .binding import (  # noqa: F401
     AstraError,
     astra_fused_add_rmsnorm,
+    astra_fused_add_rmsnorm_ex,
     astra_merge_attn_states_lse,
+    astra_merge_attn_states_lse_ex,
     astra_silu_and_mul,
+    astra_silu_and_mul_ex,
     load_library,
     status_string,
 )

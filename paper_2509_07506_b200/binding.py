@@ -31,6 +31,9 @@ EXPORTED_SYMBOLS = (
     "astra_fused_add_rmsnorm",
     "astra_silu_and_mul",
     "astra_merge_attn_states_lse",
+    "astra_fused_add_rmsnorm_ex",
+    "astra_silu_and_mul_ex",
+    "astra_merge_attn_states_lse_ex",
     "astra_status_string",
 )
 
@@ -63,6 +66,13 @@ def load_library() -> ctypes.CDLL:
     lib.astra_silu_and_mul.restype = i32
     lib.astra_merge_attn_states_lse.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, vp]
     lib.astra_merge_attn_states_lse.restype = i32
+    lib.astra_fused_add_rmsnorm_ex.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, f32, i32, vp]
+    lib.astra_fused_add_rmsnorm_ex.restype = i32
+    lib.astra_silu_and_mul_ex.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i32, vp]
+    lib.astra_silu_and_mul_ex.restype = i32
+    lib.astra_merge_attn_states_lse_ex.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64,
+                                                   ctypes.POINTER(ctypes.c_int64), i32, vp]
+    lib.astra_merge_attn_states_lse_ex.restype = i32
     lib.astra_status_string.argtypes = [i32]
     lib.astra_status_string.restype = ctypes.c_char_p
     _lib = lib
@@ -174,3 +184,93 @@ def astra_merge_attn_states_lse(v_out: torch.Tensor, lse_out: Optional[torch.Ten
             T, Hh, D, code, _stream(v_a, stream))
     if st != ASTRA_OK:
         raise AstraError(st, "astra_merge_attn_states_lse")
+
+
+# ---- strided / out-of-place forms ---------------------------------------------------------------
+
+def _check_rows(t: torch.Tensor, name: str, dtype, shape) -> None:
+    """A tensor whose innermost dimension is contiguous; outer strides are free (non-negative)."""
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    if tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} must have shape {tuple(shape)}, got {tuple(t.shape)}")
+    if t.shape[-1] > 1 and t.stride(-1) != 1:
+        raise ValueError(f"{name}: the innermost dimension must be contiguous")
+    if any(st < 0 for st in t.stride()):
+        raise ValueError(f"{name}: negative strides are not supported")
+
+
+def _pitch(t: torch.Tensor) -> int:
+    """Row pitch of a 2-D tensor (a single row may report any stride; use its width)."""
+    return t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+
+
+def astra_fused_add_rmsnorm_ex(y: torch.Tensor, residual_out: torch.Tensor, x: torch.Tensor,
+                               residual: torch.Tensor, weight: torch.Tensor, eps: float,
+                               stream: Optional[torch.cuda.Stream] = None) -> None:
+    """y <- RMSNorm(x + residual) * weight, residual_out <- x + residual; [T, H] tensors whose rows
+    may be pitched (slices of wider buffers).  y may be x and residual_out may be residual."""
+    if x.dim() != 2:
+        raise ValueError("x must be [T, H]")
+    code = _code(x, "x")
+    T, H = x.shape
+    for t, n in ((x, "x"), (residual, "residual"), (y, "y"), (residual_out, "residual_out")):
+        _check_rows(t, n, x.dtype, (T, H))
+    _check(weight, "weight", x.dtype, (H,))
+    with _on_device(x):
+        st = load_library().astra_fused_add_rmsnorm_ex(
+            y.data_ptr(), residual_out.data_ptr(), x.data_ptr(), residual.data_ptr(), weight.data_ptr(),
+            T, H, _pitch(y), _pitch(residual_out), _pitch(x), _pitch(residual), float(eps), code,
+            _stream(x, stream))
+    if st != ASTRA_OK:
+        raise AstraError(st, "astra_fused_add_rmsnorm_ex")
+
+
+def astra_silu_and_mul_ex(out: torch.Tensor, gate: torch.Tensor, up: torch.Tensor,
+                          stream: Optional[torch.cuda.Stream] = None) -> None:
+    """out[T, D] <- SiLU(gate) * up with separately addressed (possibly pitched) operands."""
+    if gate.dim() != 2:
+        raise ValueError("gate must be [T, D]")
+    code = _code(gate, "gate")
+    T, D = gate.shape
+    for t, n in ((gate, "gate"), (up, "up"), (out, "out")):
+        _check_rows(t, n, gate.dtype, (T, D))
+    with _on_device(gate):
+        st = load_library().astra_silu_and_mul_ex(out.data_ptr(), gate.data_ptr(), up.data_ptr(), T, D,
+                                                  _pitch(out), _pitch(gate), _pitch(up), code,
+                                                  _stream(gate, stream))
+    if st != ASTRA_OK:
+        raise AstraError(st, "astra_silu_and_mul_ex")
+
+
+def astra_merge_attn_states_lse_ex(v_out: torch.Tensor, lse_out: Optional[torch.Tensor],
+                                   v_a: torch.Tensor, lse_a: torch.Tensor,
+                                   v_b: torch.Tensor, lse_b: torch.Tensor,
+                                   stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Merge for strided tensors: values [T, Hh, D] with D contiguous, scores [T, Hh] with any
+    non-negative strides (e.g. the transposed view of a head-major [Hh, T] tensor)."""
+    if v_a.dim() != 3:
+        raise ValueError("v_a must be [T, Hh, D]")
+    code = _code(v_a, "v_a")
+    T, Hh, D = v_a.shape
+    for t, n in ((v_a, "v_a"), (v_b, "v_b"), (v_out, "v_out")):
+        _check_rows(t, n, v_a.dtype, (T, Hh, D))
+    scores = [(lse_a, "lse_a"), (lse_b, "lse_b")] + ([(lse_out, "lse_out")] if lse_out is not None else [])
+    for t, n in scores:
+        if not isinstance(t, torch.Tensor) or not t.is_cuda or t.dtype != torch.float32:
+            raise TypeError(f"{n} must be a float32 CUDA tensor")
+        if tuple(t.shape) != (T, Hh) or any(s < 0 for s in t.stride()):
+            raise ValueError(f"{n} must have shape {(T, Hh)} and non-negative strides")
+    so = (lse_out.stride(0), lse_out.stride(1)) if lse_out is not None else (0, 0)
+    strides = (ctypes.c_int64 * 12)(v_a.stride(0), v_a.stride(1), v_b.stride(0), v_b.stride(1),
+                                    v_out.stride(0), v_out.stride(1), lse_a.stride(0), lse_a.stride(1),
+                                    lse_b.stride(0), lse_b.stride(1), so[0], so[1])
+    with _on_device(v_a):
+        st = load_library().astra_merge_attn_states_lse_ex(
+            v_out.data_ptr(), lse_out.data_ptr() if lse_out is not None else None,
+            v_a.data_ptr(), lse_a.data_ptr(), v_b.data_ptr(), lse_b.data_ptr(), T, Hh, D, strides, code,
+            _stream(v_a, stream))
+    if st != ASTRA_OK:
+        raise AstraError(st, "astra_merge_attn_states_lse_ex")

@@ -16,24 +16,48 @@ inline bool aligned(const void *p, size_t bytes) {
     return (reinterpret_cast<uintptr_t>(p) % bytes) == 0;
 }
 
-// [a, a+na) and [b, b+nb) intersect
+// [a, a+na) and [b, b+nb) intersect (byte ranges)
 inline bool overlaps(const void *a, int64_t na, const void *b, int64_t nb) {
     const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
     return a0 < b0 + static_cast<uintptr_t>(nb) && b0 < a0 + static_cast<uintptr_t>(na);
 }
 
-// Largest vector width (in elements, up to max_vec) such that `width` is a multiple of it and every
-// pointer is aligned to it.  Rows start at multiples of `width` elements, so this makes every
-// vector access in every row aligned.
-template <typename... P>
-inline int pick_vec(int max_vec, int64_t width, P... ptrs) {
-    for (int vec = max_vec; vec > 1; vec >>= 1) {
-        if (width % vec != 0) continue;
-        const bool ok = (aligned(ptrs, static_cast<size_t>(vec) * 2) && ...);
-        if (ok) return vec;
-    }
-    return 1;
+// Bytes from the first element of a [rows, width] tensor with the given row pitch to one past its last.
+inline int64_t span_bytes(int64_t rows, int64_t width, int64_t pitch, int64_t elem) {
+    return ((rows - 1) * pitch + width) * elem;
 }
+
+// Do two [rows, width] tensors of 16-bit elements with the given row pitches share any element?
+// Exact when the pitches are equal (slices of one wider buffer: rows interleave without touching);
+// otherwise conservative (overlapping address spans count as overlap).
+inline bool pitched_overlap(const void *a, int64_t pitch_a, const void *b, int64_t pitch_b,
+                            int64_t rows, int64_t width) {
+    if (!overlaps(a, span_bytes(rows, width, pitch_a, 2), b, span_bytes(rows, width, pitch_b, 2))) return false;
+    if (pitch_a != pitch_b || rows == 1) return true;
+    const int64_t P = pitch_a * 2, w = width * 2;
+    const int64_t d = static_cast<int64_t>(reinterpret_cast<intptr_t>(b) - reinterpret_cast<intptr_t>(a));
+    int64_t k = d / P, r = d % P;  // b's row j starts r bytes into a's row j + k
+    if (r < 0) { r += P; --k; }
+    const bool hits_k = r < w && k > -rows && k < rows;
+    const bool hits_k1 = P - r < w && (k + 1) > -rows && (k + 1) < rows;
+    return hits_k || hits_k1;
+}
+
+// Largest vector width (in 16-bit elements, a power of two up to max_vec) that divides every extent
+// in `extents` and to which every pointer is aligned.  Row starts are multiples of the pitches, so
+// every vector access of every row is then naturally aligned.
+struct VecPick {
+    int vec;
+    explicit VecPick(int max_vec) : vec(max_vec) {}
+    VecPick &extent(int64_t e) {
+        while (vec > 1 && e % vec != 0) vec >>= 1;
+        return *this;
+    }
+    VecPick &pointer(const void *p) {
+        while (vec > 1 && !aligned(p, static_cast<size_t>(vec) * 2)) vec >>= 1;
+        return *this;
+    }
+};
 
 inline astra_status_t launch_status() {
     return cudaGetLastError() == cudaSuccess ? ASTRA_OK : ASTRA_ERR_CUDA;
@@ -60,12 +84,16 @@ inline void launch(void (*kernel)(KArgs...), unsigned grid, unsigned block, cuda
 }
 
 constexpr int64_t kMaxVecsPerLaunch = (1ll << 31) - 1;  // flat vector indices are 31-bit
+constexpr int64_t kInt64Max = 9223372036854775807ll;
+
+inline bool valid_dtype(astra_dtype_t d) { return d == ASTRA_BF16 || d == ASTRA_FP16; }
 
 // ---------------------------------------------------------------------------------------------
 // silu_and_mul
 // ---------------------------------------------------------------------------------------------
 template <int DT, int VEC, int UNROLL, int THREADS>
-void launch_silu(uint16_t *out, const uint16_t *in, int64_t T, int64_t D, cudaStream_t stream) {
+void launch_silu(uint16_t *out, const uint16_t *gate, const uint16_t *up, int64_t T, int64_t D,
+                 int64_t out_pitch, int64_t gate_pitch, int64_t up_pitch, cudaStream_t stream) {
     const int64_t nvec = D / VEC;
     const int64_t rows_per_launch = kMaxVecsPerLaunch / nvec;
     for (int64_t t0 = 0; t0 < T; t0 += rows_per_launch) {
@@ -74,21 +102,49 @@ void launch_silu(uint16_t *out, const uint16_t *in, int64_t T, int64_t D, cudaSt
         const uint32_t tile = THREADS * UNROLL;
         const uint32_t blocks = (total + tile - 1) / tile;
         launch(silu_and_mul_kernel<DT, VEC, UNROLL, THREADS>, blocks, THREADS, stream,
-               out + t0 * D, in + t0 * 2 * D, total, FastDiv::make(static_cast<uint32_t>(nvec)), D);
+               out + t0 * out_pitch, gate + t0 * gate_pitch, up + t0 * up_pitch, total,
+               FastDiv::make(static_cast<uint32_t>(nvec)), out_pitch, gate_pitch, up_pitch);
     }
 }
 
 template <int DT>
-void dispatch_silu(uint16_t *out, const uint16_t *in, int64_t T, int64_t D, cudaStream_t stream) {
-    // each row is [a | b]: a starts at 2*D*t and b at 2*D*t + D, so D itself must be a multiple of VEC
+void dispatch_silu(uint16_t *out, const uint16_t *gate, const uint16_t *up, int64_t T, int64_t D,
+                   int64_t out_pitch, int64_t gate_pitch, int64_t up_pitch, cudaStream_t stream) {
+    const int vec = VecPick(8).extent(D).extent(out_pitch).extent(gate_pitch).extent(up_pitch)
+                        .pointer(out).pointer(gate).pointer(up).vec;
     // One 16-byte vector per thread and 256-thread blocks: the smallest work quantum that still
     // keeps the block scheduler ahead, which gives the shortest drain at the end of the grid.
-    switch (pick_vec(8, D, out, in)) {
-        case 8: launch_silu<DT, 8, 1, 256>(out, in, T, D, stream); break;
-        case 4: launch_silu<DT, 4, 4, 256>(out, in, T, D, stream); break;
-        case 2: launch_silu<DT, 2, 4, 256>(out, in, T, D, stream); break;
-        default: launch_silu<DT, 1, 4, 256>(out, in, T, D, stream); break;
+    switch (vec) {
+        case 8: launch_silu<DT, 8, 1, 256>(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, stream); break;
+        case 4: launch_silu<DT, 4, 4, 256>(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, stream); break;
+        case 2: launch_silu<DT, 2, 4, 256>(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, stream); break;
+        default: launch_silu<DT, 1, 4, 256>(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, stream); break;
     }
+}
+
+astra_status_t silu_entry(void *out, const void *gate, const void *up, int64_t T, int64_t D,
+                          int64_t out_pitch, int64_t gate_pitch, int64_t up_pitch,
+                          astra_dtype_t dtype, void *cuda_stream) {
+    if (!out || !gate || !up) return ASTRA_ERR_NULL_POINTER;
+    if (!valid_dtype(dtype)) return ASTRA_ERR_BAD_DTYPE;
+    if (T < 0 || D <= 0 || D > 1073741823ll) return ASTRA_ERR_BAD_SHAPE;
+    if (out_pitch < D || gate_pitch < D || up_pitch < D) return ASTRA_ERR_BAD_SHAPE;
+    const int64_t max_pitch = out_pitch > gate_pitch ? (out_pitch > up_pitch ? out_pitch : up_pitch)
+                                                     : (gate_pitch > up_pitch ? gate_pitch : up_pitch);
+    if (T > 0 && max_pitch > kInt64Max / 4 / T) return ASTRA_ERR_BAD_SHAPE;
+    if (!aligned(out, 2) || !aligned(gate, 2) || !aligned(up, 2)) return ASTRA_ERR_MISALIGNED;
+    if (T == 0) return ASTRA_OK;
+    if (pitched_overlap(out, out_pitch, gate, gate_pitch, T, D) ||
+        pitched_overlap(out, out_pitch, up, up_pitch, T, D))
+        return ASTRA_ERR_OVERLAP;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint16_t *op = static_cast<uint16_t *>(out);
+    const uint16_t *gp = static_cast<const uint16_t *>(gate), *upp = static_cast<const uint16_t *>(up);
+    if (dtype == ASTRA_BF16)
+        dispatch_silu<ASTRA_BF16>(op, gp, upp, T, D, out_pitch, gate_pitch, up_pitch, stream);
+    else
+        dispatch_silu<ASTRA_FP16>(op, gp, upp, T, D, out_pitch, gate_pitch, up_pitch, stream);
+    return launch_status();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -115,7 +171,8 @@ template <int DT>
 void dispatch_merge(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
                     const uint16_t *v_b, const float *lse_b, int64_t rows, int64_t D,
                     cudaStream_t stream) {
-    switch (pick_vec(16, D, v_out, v_a, v_b)) {
+    // 32-byte accesses measured best here (one per thread, 256-thread blocks)
+    switch (VecPick(16).extent(D).pointer(v_out).pointer(v_a).pointer(v_b).vec) {
         case 16: launch_merge<DT, 16, 1, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream); break;
         case 8: launch_merge<DT, 8, 2, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream); break;
         case 4: launch_merge<DT, 4, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream); break;
@@ -124,19 +181,74 @@ void dispatch_merge(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const 
     }
 }
 
+template <int DT, int VEC, int UNROLL, int THREADS>
+void launch_merge_strided(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
+                          const uint16_t *v_b, const float *lse_b, int64_t rows_total, int64_t Hh,
+                          int64_t D, const MergeStrides &st, cudaStream_t stream) {
+    const int64_t nvec = D / VEC;
+    const int64_t rows_per_launch = kMaxVecsPerLaunch / nvec;
+    for (int64_t r0 = 0; r0 < rows_total; r0 += rows_per_launch) {
+        const int64_t rows = (rows_total - r0 < rows_per_launch) ? (rows_total - r0) : rows_per_launch;
+        const uint32_t total = static_cast<uint32_t>(rows * nvec);
+        const uint32_t tile = THREADS * UNROLL;
+        const uint32_t blocks = (total + tile - 1) / tile;
+        launch(merge_attn_states_lse_strided_kernel<DT, VEC, UNROLL, THREADS>, blocks, THREADS, stream,
+               v_out, lse_out, v_a, lse_a, v_b, lse_b, total, static_cast<uint32_t>(r0),
+               FastDiv::make(static_cast<uint32_t>(nvec)), FastDiv::make(static_cast<uint32_t>(Hh)), st);
+    }
+}
+
+template <int DT>
+void dispatch_merge_strided(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
+                            const uint16_t *v_b, const float *lse_b, int64_t rows, int64_t Hh, int64_t D,
+                            const MergeStrides &st, cudaStream_t stream) {
+    const int vec = VecPick(16).extent(D).extent(st.va_t).extent(st.va_h).extent(st.vb_t).extent(st.vb_h)
+                        .extent(st.vo_t).extent(st.vo_h).pointer(v_out).pointer(v_a).pointer(v_b).vec;
+    switch (vec) {
+        case 16: launch_merge_strided<DT, 16, 1, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, Hh, D, st, stream); break;
+        case 8: launch_merge_strided<DT, 8, 2, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, Hh, D, st, stream); break;
+        case 4: launch_merge_strided<DT, 4, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, Hh, D, st, stream); break;
+        case 2: launch_merge_strided<DT, 2, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, Hh, D, st, stream); break;
+        default: launch_merge_strided<DT, 1, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, Hh, D, st, stream); break;
+    }
+}
+
+// One past the largest element offset of a [T, Hh, W] tensor addressed by (token, head) strides.
+inline int64_t strided_extent(int64_t T, int64_t Hh, int64_t W, int64_t st, int64_t sh) {
+    return (T - 1) * st + (Hh - 1) * sh + W;
+}
+
+// The (token, head) rows of W contiguous elements must not overlap one another: with the smaller
+// stride s1 over n1 steps and the larger s2, require s1 >= W (or n1 == 1) and s2 >= extent of the
+// inner dimension (or n2 == 1).
+inline bool rows_disjoint(int64_t T, int64_t Hh, int64_t W, int64_t st, int64_t sh) {
+    int64_t n1 = Hh, s1 = sh, n2 = T, s2 = st;
+    if ((n1 > 1 && n2 > 1 && s1 > s2) || n1 == 1) {
+        int64_t tn = n1, ts = s1;
+        n1 = n2; s1 = s2; n2 = tn; s2 = ts;
+    }
+    if (n1 > 1 && s1 < W) return false;
+    if (n2 > 1 && s2 < (n1 - 1) * s1 + W) return false;
+    return true;
+}
+
 // ---------------------------------------------------------------------------------------------
 // fused_add_rmsnorm
 // ---------------------------------------------------------------------------------------------
 constexpr int kMaxGridX = 2147483647;
 
+// Most elements of a row one thread keeps in registers: 64 with vector accesses, 16 on the scalar
+// path (each element then also costs three separate packed-input registers).
+constexpr int rmsnorm_max_elems_per_thread(int vec) { return vec == 1 ? 16 : 64; }
+
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 template <int DT, int VEC, int VPT>
-inline void launch_rmsnorm_reg(unsigned rows, int threads, cudaStream_t stream, uint16_t *x, uint16_t *r,
+inline void launch_rmsnorm_reg(unsigned rows, int threads, cudaStream_t stream, const RmsnormOperands &op,
                                const uint16_t *w, int H, float eps, float inv_H) {
-    // at most 64 elements per thread are ever selected; wider combinations are not instantiated
-    if constexpr (VEC * VPT <= 64)
-        launch(fused_add_rmsnorm_reg_kernel<DT, VEC, VPT>, rows, threads, stream, x, r, w, H, eps, inv_H);
+    // wider combinations than the per-thread cap are never selected and are not instantiated
+    if constexpr (VEC * VPT <= rmsnorm_max_elems_per_thread(VEC))
+        launch(fused_add_rmsnorm_reg_kernel<DT, VEC, VPT>, rows, threads, stream, op, w, H, eps, inv_H);
 }
 
 // Register-resident rows: VPT vectors per thread with blockDim = ceil(nvec / VPT) rounded up to a warp.
@@ -144,49 +256,99 @@ inline void launch_rmsnorm_reg(unsigned rows, int threads, cudaStream_t stream, 
 // measured best; up to 64 elements per thread are used for wider rows, with the block size capped
 // so the row still fits the register file.  Rows wider than that take the two-sweep kernel.
 template <int DT, int VEC>
-void launch_rmsnorm(uint16_t *x, uint16_t *r, const uint16_t *w, int64_t T, int H, float eps,
-                    cudaStream_t stream) {
+void launch_rmsnorm(RmsnormOperands op, const uint16_t *w, int64_t T, int H, float eps, cudaStream_t stream) {
     const int nvec = H / VEC;
     const float inv_H = 1.0f / static_cast<float>(H);
     // start at 16 elements per thread; widen the per-thread share only if the row needs more
     // threads than that share allows, narrow it if the block would fall under 128 threads
     int vpt = 16 / VEC < 1 ? 1 : 16 / VEC;
     auto threads_for = [&](int v) { return round_up((nvec + v - 1) / v, 32); };
-    while (vpt < 64 / VEC && threads_for(vpt) > rmsnorm_reg_max_threads(VEC, vpt)) vpt <<= 1;
+    while (vpt < rmsnorm_max_elems_per_thread(VEC) / VEC && threads_for(vpt) > rmsnorm_reg_max_threads(VEC, vpt)) vpt <<= 1;
     while (vpt > 1 && threads_for(vpt) < 128) vpt >>= 1;
     const int threads = threads_for(vpt);
     const bool fits = threads <= rmsnorm_reg_max_threads(VEC, vpt);
     for (int64_t t0 = 0; t0 < T; t0 += kMaxGridX) {
         const unsigned rows = static_cast<unsigned>(T - t0 < kMaxGridX ? T - t0 : kMaxGridX);
-        uint16_t *xs = x + t0 * H, *rs = r + t0 * H;
+        RmsnormOperands o = op;
+        o.x += t0 * op.x_pitch;
+        o.r += t0 * op.r_pitch;
+        o.y += t0 * op.y_pitch;
+        o.r_out += t0 * op.r_out_pitch;
         if (!fits) {
-            launch(fused_add_rmsnorm_twopass_kernel<DT, VEC>, rows, 1024, stream, xs, rs, w, H, eps, inv_H);
+            launch(fused_add_rmsnorm_twopass_kernel<DT, VEC>, rows, 1024, stream, o, w, H, eps, inv_H);
             continue;
         }
         switch (vpt) {
-            case 1: launch_rmsnorm_reg<DT, VEC, 1>(rows, threads, stream, xs, rs, w, H, eps, inv_H); break;
-            case 2: launch_rmsnorm_reg<DT, VEC, 2>(rows, threads, stream, xs, rs, w, H, eps, inv_H); break;
-            case 4: launch_rmsnorm_reg<DT, VEC, 4>(rows, threads, stream, xs, rs, w, H, eps, inv_H); break;
-            case 8: launch_rmsnorm_reg<DT, VEC, 8>(rows, threads, stream, xs, rs, w, H, eps, inv_H); break;
-            case 16: launch_rmsnorm_reg<DT, VEC, 16>(rows, threads, stream, xs, rs, w, H, eps, inv_H); break;
-            case 32: launch_rmsnorm_reg<DT, VEC, 32>(rows, threads, stream, xs, rs, w, H, eps, inv_H); break;
-            default: launch_rmsnorm_reg<DT, VEC, 64>(rows, threads, stream, xs, rs, w, H, eps, inv_H); break;
+            case 1: launch_rmsnorm_reg<DT, VEC, 1>(rows, threads, stream, o, w, H, eps, inv_H); break;
+            case 2: launch_rmsnorm_reg<DT, VEC, 2>(rows, threads, stream, o, w, H, eps, inv_H); break;
+            case 4: launch_rmsnorm_reg<DT, VEC, 4>(rows, threads, stream, o, w, H, eps, inv_H); break;
+            case 8: launch_rmsnorm_reg<DT, VEC, 8>(rows, threads, stream, o, w, H, eps, inv_H); break;
+            case 16: launch_rmsnorm_reg<DT, VEC, 16>(rows, threads, stream, o, w, H, eps, inv_H); break;
+            case 32: launch_rmsnorm_reg<DT, VEC, 32>(rows, threads, stream, o, w, H, eps, inv_H); break;
+            default: launch_rmsnorm_reg<DT, VEC, 64>(rows, threads, stream, o, w, H, eps, inv_H); break;
         }
     }
 }
 
 template <int DT>
-void dispatch_rmsnorm(uint16_t *x, uint16_t *r, const uint16_t *w, int64_t T, int H, float eps,
+void dispatch_rmsnorm(const RmsnormOperands &op, const uint16_t *w, int64_t T, int H, float eps,
                       cudaStream_t stream) {
-    switch (pick_vec(8, H, x, r, w)) {
-        case 8: launch_rmsnorm<DT, 8>(x, r, w, T, H, eps, stream); break;
-        case 4: launch_rmsnorm<DT, 4>(x, r, w, T, H, eps, stream); break;
-        case 2: launch_rmsnorm<DT, 2>(x, r, w, T, H, eps, stream); break;
-        default: launch_rmsnorm<DT, 1>(x, r, w, T, H, eps, stream); break;
+    const int vec = VecPick(8).extent(H).extent(op.x_pitch).extent(op.r_pitch).extent(op.y_pitch)
+                        .extent(op.r_out_pitch).pointer(op.x).pointer(op.r).pointer(op.y).pointer(op.r_out)
+                        .pointer(w).vec;
+    switch (vec) {
+        case 8: launch_rmsnorm<DT, 8>(op, w, T, H, eps, stream); break;
+        case 4: launch_rmsnorm<DT, 4>(op, w, T, H, eps, stream); break;
+        case 2: launch_rmsnorm<DT, 2>(op, w, T, H, eps, stream); break;
+        default: launch_rmsnorm<DT, 1>(op, w, T, H, eps, stream); break;
     }
 }
 
-inline bool valid_dtype(astra_dtype_t d) { return d == ASTRA_BF16 || d == ASTRA_FP16; }
+astra_status_t rmsnorm_entry(void *y, void *residual_out, const void *x, const void *residual,
+                             const void *weight, int64_t T, int64_t H, int64_t y_pitch,
+                             int64_t ro_pitch, int64_t x_pitch, int64_t r_pitch, float eps,
+                             astra_dtype_t dtype, void *cuda_stream) {
+    if (!y || !residual_out || !x || !residual || !weight) return ASTRA_ERR_NULL_POINTER;
+    if (!valid_dtype(dtype)) return ASTRA_ERR_BAD_DTYPE;
+    if (T < 0 || H <= 0 || H > 2147483647ll) return ASTRA_ERR_BAD_SHAPE;
+    if (y_pitch < H || ro_pitch < H || x_pitch < H || r_pitch < H) return ASTRA_ERR_BAD_SHAPE;
+    int64_t max_pitch = y_pitch;
+    if (ro_pitch > max_pitch) max_pitch = ro_pitch;
+    if (x_pitch > max_pitch) max_pitch = x_pitch;
+    if (r_pitch > max_pitch) max_pitch = r_pitch;
+    if (T > 0 && max_pitch > kInt64Max / 4 / T) return ASTRA_ERR_BAD_SHAPE;
+    if (!aligned(y, 2) || !aligned(residual_out, 2) || !aligned(x, 2) || !aligned(residual, 2) ||
+        !aligned(weight, 2))
+        return ASTRA_ERR_MISALIGNED;
+    if (T == 0) return ASTRA_OK;
+    const bool y_is_x = (y == x && y_pitch == x_pitch);
+    const bool ro_is_r = (residual_out == residual && ro_pitch == r_pitch);
+    // the weight is one row: compare it against every output as a [T, H] tensor of pitch 0 would be
+    // wrong (pitch < width), so use the outputs' spans for it
+    const int64_t sy = span_bytes(T, H, y_pitch, 2), sro = span_bytes(T, H, ro_pitch, 2), sw = H * 2;
+    if ((!y_is_x && pitched_overlap(y, y_pitch, x, x_pitch, T, H)) ||
+        pitched_overlap(y, y_pitch, residual, r_pitch, T, H) ||
+        pitched_overlap(y, y_pitch, residual_out, ro_pitch, T, H) || overlaps(y, sy, weight, sw) ||
+        (!ro_is_r && pitched_overlap(residual_out, ro_pitch, residual, r_pitch, T, H)) ||
+        pitched_overlap(residual_out, ro_pitch, x, x_pitch, T, H) || overlaps(residual_out, sro, weight, sw))
+        return ASTRA_ERR_OVERLAP;
+    RmsnormOperands op;
+    op.x = static_cast<const uint16_t *>(x);
+    op.r = static_cast<const uint16_t *>(residual);
+    op.y = static_cast<uint16_t *>(y);
+    op.r_out = static_cast<uint16_t *>(residual_out);
+    op.x_pitch = x_pitch;
+    op.r_pitch = r_pitch;
+    op.y_pitch = y_pitch;
+    op.r_out_pitch = ro_pitch;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const uint16_t *wp = static_cast<const uint16_t *>(weight);
+    if (dtype == ASTRA_BF16)
+        dispatch_rmsnorm<ASTRA_BF16>(op, wp, T, static_cast<int>(H), eps, stream);
+    else
+        dispatch_rmsnorm<ASTRA_FP16>(op, wp, T, static_cast<int>(H), eps, stream);
+    return launch_status();
+}
 
 }  // namespace
 
@@ -194,43 +356,30 @@ extern "C" {
 
 astra_status_t astra_fused_add_rmsnorm(void *x, void *residual, const void *weight, int64_t T,
                                        int64_t H, float eps, astra_dtype_t dtype, void *cuda_stream) {
-    if (!x || !residual || !weight) return ASTRA_ERR_NULL_POINTER;
-    if (!valid_dtype(dtype)) return ASTRA_ERR_BAD_DTYPE;
-    if (T < 0 || H <= 0 || H > 2147483647ll) return ASTRA_ERR_BAD_SHAPE;
-    if (T > 0 && H > INT64_MAX / 2 / T) return ASTRA_ERR_BAD_SHAPE;
-    if (!aligned(x, 2) || !aligned(residual, 2) || !aligned(weight, 2)) return ASTRA_ERR_MISALIGNED;
-    if (T == 0) return ASTRA_OK;
-    const int64_t bytes = T * H * 2;
-    if (overlaps(x, bytes, residual, bytes) || overlaps(x, bytes, weight, H * 2) ||
-        overlaps(residual, bytes, weight, H * 2))
-        return ASTRA_ERR_OVERLAP;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    uint16_t *xp = static_cast<uint16_t *>(x), *rp = static_cast<uint16_t *>(residual);
-    const uint16_t *wp = static_cast<const uint16_t *>(weight);
-    if (dtype == ASTRA_BF16)
-        dispatch_rmsnorm<ASTRA_BF16>(xp, rp, wp, T, static_cast<int>(H), eps, stream);
-    else
-        dispatch_rmsnorm<ASTRA_FP16>(xp, rp, wp, T, static_cast<int>(H), eps, stream);
-    return launch_status();
+    return rmsnorm_entry(x, residual, x, residual, weight, T, H, H, H, H, H, eps, dtype, cuda_stream);
+}
+
+astra_status_t astra_fused_add_rmsnorm_ex(void *y, void *residual_out, const void *x,
+                                          const void *residual, const void *weight, int64_t T,
+                                          int64_t H, int64_t y_pitch, int64_t residual_out_pitch,
+                                          int64_t x_pitch, int64_t residual_pitch, float eps,
+                                          astra_dtype_t dtype, void *cuda_stream) {
+    return rmsnorm_entry(y, residual_out, x, residual, weight, T, H, y_pitch, residual_out_pitch,
+                         x_pitch, residual_pitch, eps, dtype, cuda_stream);
 }
 
 astra_status_t astra_silu_and_mul(void *out, const void *input, int64_t T, int64_t D,
                                   astra_dtype_t dtype, void *cuda_stream) {
-    if (!out || !input) return ASTRA_ERR_NULL_POINTER;
-    if (!valid_dtype(dtype)) return ASTRA_ERR_BAD_DTYPE;
-    if (T < 0 || D <= 0 || D > 1073741823ll) return ASTRA_ERR_BAD_SHAPE;
-    if (T > 0 && D > INT64_MAX / 4 / T) return ASTRA_ERR_BAD_SHAPE;
-    if (!aligned(out, 2) || !aligned(input, 2)) return ASTRA_ERR_MISALIGNED;
-    if (T == 0) return ASTRA_OK;
-    if (overlaps(out, T * D * 2, input, T * D * 4)) return ASTRA_ERR_OVERLAP;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    uint16_t *op = static_cast<uint16_t *>(out);
-    const uint16_t *ip = static_cast<const uint16_t *>(input);
-    if (dtype == ASTRA_BF16)
-        dispatch_silu<ASTRA_BF16>(op, ip, T, D, stream);
-    else
-        dispatch_silu<ASTRA_FP16>(op, ip, T, D, stream);
-    return launch_status();
+    if (!input) return ASTRA_ERR_NULL_POINTER;
+    if (D <= 0 || D > 1073741823ll) return ASTRA_ERR_BAD_SHAPE;
+    const void *up = static_cast<const uint16_t *>(input) + D;
+    return silu_entry(out, input, up, T, D, D, 2 * D, 2 * D, dtype, cuda_stream);
+}
+
+astra_status_t astra_silu_and_mul_ex(void *out, const void *gate, const void *up, int64_t T,
+                                     int64_t D, int64_t out_pitch, int64_t gate_pitch,
+                                     int64_t up_pitch, astra_dtype_t dtype, void *cuda_stream) {
+    return silu_entry(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, dtype, cuda_stream);
 }
 
 astra_status_t astra_merge_attn_states_lse(void *v_out, float *lse_out, const void *v_a,
@@ -240,7 +389,7 @@ astra_status_t astra_merge_attn_states_lse(void *v_out, float *lse_out, const vo
     if (!v_out || !v_a || !v_b || !lse_a || !lse_b) return ASTRA_ERR_NULL_POINTER;
     if (!valid_dtype(dtype)) return ASTRA_ERR_BAD_DTYPE;
     if (T < 0 || Hh <= 0 || D <= 0 || D > 2147483647ll) return ASTRA_ERR_BAD_SHAPE;
-    if (T > 0 && (Hh > INT64_MAX / 4 / T || D > INT64_MAX / 4 / (T * Hh))) return ASTRA_ERR_BAD_SHAPE;
+    if (T > 0 && (Hh > kInt64Max / 4 / T || D > kInt64Max / 4 / (T * Hh))) return ASTRA_ERR_BAD_SHAPE;
     if (!aligned(v_out, 2) || !aligned(v_a, 2) || !aligned(v_b, 2) || !aligned(lse_a, 4) ||
         !aligned(lse_b, 4) || (lse_out && !aligned(lse_out, 4)))
         return ASTRA_ERR_MISALIGNED;
@@ -263,6 +412,59 @@ astra_status_t astra_merge_attn_states_lse(void *v_out, float *lse_out, const vo
         dispatch_merge<ASTRA_BF16>(vo, lse_out, va, lse_a, vb, lse_b, rows, D, stream);
     else
         dispatch_merge<ASTRA_FP16>(vo, lse_out, va, lse_a, vb, lse_b, rows, D, stream);
+    return launch_status();
+}
+
+astra_status_t astra_merge_attn_states_lse_ex(void *v_out, float *lse_out, const void *v_a,
+                                              const float *lse_a, const void *v_b, const float *lse_b,
+                                              int64_t T, int64_t Hh, int64_t D, const int64_t *strides,
+                                              astra_dtype_t dtype, void *cuda_stream) {
+    if (!v_out || !v_a || !v_b || !lse_a || !lse_b || !strides) return ASTRA_ERR_NULL_POINTER;
+    if (!valid_dtype(dtype)) return ASTRA_ERR_BAD_DTYPE;
+    if (T < 0 || Hh <= 0 || D <= 0 || D > 2147483647ll || Hh > 2147483647ll) return ASTRA_ERR_BAD_SHAPE;
+    if (T > 0 && T * Hh > 2147483647ll) return ASTRA_ERR_BAD_SHAPE;
+    for (int i = 0; i < 12; ++i) {
+        if (lse_out == nullptr && i >= 10) break;
+        // every offset (T-1)*stride, (Hh-1)*stride must stay far inside int64
+        const int64_t steps = (i % 2 == 0 ? T : Hh) - 1;
+        if (strides[i] < 0 || (steps > 0 && strides[i] > (1ll << 60) / steps)) return ASTRA_ERR_BAD_SHAPE;
+    }
+    MergeStrides st;
+    st.va_t = strides[0]; st.va_h = strides[1]; st.vb_t = strides[2]; st.vb_h = strides[3];
+    st.vo_t = strides[4]; st.vo_h = strides[5]; st.sa_t = strides[6]; st.sa_h = strides[7];
+    st.sb_t = strides[8]; st.sb_h = strides[9];
+    st.so_t = lse_out ? strides[10] : 0;
+    st.so_h = lse_out ? strides[11] : 0;
+    if (!aligned(v_out, 2) || !aligned(v_a, 2) || !aligned(v_b, 2) || !aligned(lse_a, 4) ||
+        !aligned(lse_b, 4) || (lse_out && !aligned(lse_out, 4)))
+        return ASTRA_ERR_MISALIGNED;
+    if (T == 0) return ASTRA_OK;
+    // written tensors must have non-overlapping rows; read tensors may broadcast (stride 0)
+    if (!rows_disjoint(T, Hh, D, st.vo_t, st.vo_h)) return ASTRA_ERR_BAD_SHAPE;
+    if (lse_out && !rows_disjoint(T, Hh, 1, st.so_t, st.so_h)) return ASTRA_ERR_BAD_SHAPE;
+    const int64_t bva = strided_extent(T, Hh, D, st.va_t, st.va_h) * 2;
+    const int64_t bvb = strided_extent(T, Hh, D, st.vb_t, st.vb_h) * 2;
+    const int64_t bvo = strided_extent(T, Hh, D, st.vo_t, st.vo_h) * 2;
+    const int64_t bsa = strided_extent(T, Hh, 1, st.sa_t, st.sa_h) * 4;
+    const int64_t bsb = strided_extent(T, Hh, 1, st.sb_t, st.sb_h) * 4;
+    const int64_t bso = lse_out ? strided_extent(T, Hh, 1, st.so_t, st.so_h) * 4 : 0;
+    const bool out_is_a = (v_out == v_a && st.vo_t == st.va_t && st.vo_h == st.va_h);
+    const bool out_is_b = (v_out == v_b && st.vo_t == st.vb_t && st.vo_h == st.vb_h);
+    if ((!out_is_a && overlaps(v_out, bvo, v_a, bva)) || (!out_is_b && overlaps(v_out, bvo, v_b, bvb)) ||
+        overlaps(v_out, bvo, lse_a, bsa) || overlaps(v_out, bvo, lse_b, bsb))
+        return ASTRA_ERR_OVERLAP;
+    if (lse_out && (overlaps(lse_out, bso, lse_a, bsa) || overlaps(lse_out, bso, lse_b, bsb) ||
+                    overlaps(lse_out, bso, v_a, bva) || overlaps(lse_out, bso, v_b, bvb) ||
+                    overlaps(lse_out, bso, v_out, bvo)))
+        return ASTRA_ERR_OVERLAP;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint16_t *vo = static_cast<uint16_t *>(v_out);
+    const uint16_t *va = static_cast<const uint16_t *>(v_a), *vb = static_cast<const uint16_t *>(v_b);
+    const int64_t rows = T * Hh;
+    if (dtype == ASTRA_BF16)
+        dispatch_merge_strided<ASTRA_BF16>(vo, lse_out, va, lse_a, vb, lse_b, rows, Hh, D, st, stream);
+    else
+        dispatch_merge_strided<ASTRA_FP16>(vo, lse_out, va, lse_a, vb, lse_b, rows, Hh, D, st, stream);
     return launch_status();
 }
 

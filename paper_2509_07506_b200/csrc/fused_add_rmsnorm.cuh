@@ -1,5 +1,6 @@
 // fused_add_rmsnorm (Astra paper, Table 1, Kernel 2):
-//     s = x + r;   r <- s;   x <- s / sqrt(mean(s^2) + eps) * w        per row of H elements.
+//     s = x + r;   r_out <- s;   y <- s / sqrt(mean(s^2) + eps) * w        per row of H elements
+// (in place when y is x and r_out is r).
 //
 // HBM-bound: 8 bytes move per element (x and r read once, y and the new r written once).  One
 // thread block owns one row.  In the register-resident kernel each thread keeps its share of the
@@ -14,6 +15,16 @@
 namespace astra {
 
 constexpr int kMaxWarps = 32;
+
+// Row-addressed operands.  Pitches are in elements.  y may be exactly x and r_out exactly r (the
+// in-place form); each thread reads the vectors it later overwrites, so that aliasing is safe.
+struct RmsnormOperands {
+    const uint16_t *x;
+    const uint16_t *r;
+    uint16_t *y;
+    uint16_t *r_out;
+    int64_t x_pitch, r_pitch, y_pitch, r_out_pitch;
+};
 
 // Sum over the block; every thread receives the total.  `slots` holds kMaxWarps floats.
 __device__ __forceinline__ float block_sum(float v, float *slots) {
@@ -40,14 +51,15 @@ __host__ __device__ constexpr int rmsnorm_reg_max_threads(int vec, int vpt) {
 // Requires nvec = H / VEC <= VPT * blockDim.x and blockDim.x <= rmsnorm_reg_max_threads(VEC, VPT).
 template <int DT, int VEC, int VPT, Ld LDH = Ld::Stream, St STH = St::Stream>
 __global__ void __launch_bounds__(rmsnorm_reg_max_threads(VEC, VPT))
-fused_add_rmsnorm_reg_kernel(uint16_t *x, uint16_t *residual,
-                                             const uint16_t *__restrict__ weight,
-                                             int H, float eps, float inv_H) {
+fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ weight,
+                             int H, float eps, float inv_H) {
     __shared__ float slots[kMaxWarps];
     const int nvec = H / VEC;
-    const int64_t row_off = static_cast<int64_t>(blockIdx.x) * H;
-    uint16_t *xr = x + row_off;
-    uint16_t *rr = residual + row_off;
+    const int64_t row = blockIdx.x;
+    const uint16_t *xr = op.x + row * op.x_pitch;
+    const uint16_t *rr = op.r + row * op.r_pitch;
+    uint16_t *yr = op.y + row * op.y_pitch;
+    uint16_t *ror = op.r_out + row * op.r_out_pitch;
     grid_dependency_wait();
     grid_launch_dependents();
 
@@ -56,7 +68,7 @@ fused_add_rmsnorm_reg_kernel(uint16_t *x, uint16_t *residual,
     for (int i = 0; i < VPT; ++i) {
         const int v = threadIdx.x + i * blockDim.x;
         if (v < nvec) {
-            // x and residual are rewritten by this same thread below: coherent loads, not .nc
+            // x and residual may be rewritten by this same thread below: coherent loads, not .nc
             px[i] = load<VEC, LDH>(xr + v * VEC);
             pr[i] = load<VEC, LDH>(rr + v * VEC);
         }
@@ -81,7 +93,7 @@ fused_add_rmsnorm_reg_kernel(uint16_t *x, uint16_t *residual,
                 s[i][k] = fx[k] + fr[k];  // the one binary32 add
                 acc = fmaf(s[i][k], s[i][k], acc);
             }
-            store<VEC, STH>(rr + v * VEC, narrow<DT, VEC>(s[i]));
+            store<VEC, STH>(ror + v * VEC, narrow<DT, VEC>(s[i]));
         }
     }
 
@@ -96,7 +108,7 @@ fused_add_rmsnorm_reg_kernel(uint16_t *x, uint16_t *residual,
             widen<DT, VEC>(pw[i], fw);
 #pragma unroll
             for (int k = 0; k < VEC; ++k) fy[k] = s[i][k] * rstd * fw[k];
-            store<VEC, STH>(xr + v * VEC, narrow<DT, VEC>(fy));
+            store<VEC, STH>(yr + v * VEC, narrow<DT, VEC>(fy));
         }
     }
 }
@@ -106,14 +118,16 @@ fused_add_rmsnorm_reg_kernel(uint16_t *x, uint16_t *residual,
 // binary32 sums, and writes both outputs.  Nothing is written before the norm is known, so the
 // in-place update cannot disturb the reduction.
 template <int DT, int VEC>
-__global__ void fused_add_rmsnorm_twopass_kernel(uint16_t *x, uint16_t *residual,
+__global__ void fused_add_rmsnorm_twopass_kernel(RmsnormOperands op,
                                                  const uint16_t *__restrict__ weight,
                                                  int H, float eps, float inv_H) {
     __shared__ float slots[kMaxWarps];
     const int nvec = H / VEC;
-    const int64_t row_off = static_cast<int64_t>(blockIdx.x) * H;
-    uint16_t *xr = x + row_off;
-    uint16_t *rr = residual + row_off;
+    const int64_t row = blockIdx.x;
+    const uint16_t *xr = op.x + row * op.x_pitch;
+    const uint16_t *rr = op.r + row * op.r_pitch;
+    uint16_t *yr = op.y + row * op.y_pitch;
+    uint16_t *ror = op.r_out + row * op.r_out_pitch;
     grid_dependency_wait();
     grid_launch_dependents();
 
@@ -141,8 +155,8 @@ __global__ void fused_add_rmsnorm_twopass_kernel(uint16_t *x, uint16_t *residual
             fs[k] = fx[k] + fr[k];
             fy[k] = fs[k] * rstd * fw[k];
         }
-        store<VEC, St::Stream>(rr + v * VEC, narrow<DT, VEC>(fs));
-        store<VEC, St::Stream>(xr + v * VEC, narrow<DT, VEC>(fy));
+        store<VEC, St::Stream>(ror + v * VEC, narrow<DT, VEC>(fs));
+        store<VEC, St::Stream>(yr + v * VEC, narrow<DT, VEC>(fy));
     }
 }
 

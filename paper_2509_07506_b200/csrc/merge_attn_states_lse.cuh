@@ -48,6 +48,12 @@ __device__ __forceinline__ MergeWeights merge_weights(float sa, float sb) {
     return r;
 }
 
+// Strides (in elements) of one [T, Hh, D] value tensor or one [T, Hh] score tensor; D is contiguous.
+struct MergeStrides {
+    int64_t va_t, va_h, vb_t, vb_h, vo_t, vo_h;  // values: token and head strides
+    int64_t sa_t, sa_h, sb_t, sb_h, so_t, so_h;  // scores: token and head strides
+};
+
 // Flat indexing over vectors of VEC elements: vector v belongs to row = v / nvec (row = token*Hh+head).
 template <int DT, int VEC, int UNROLL, int THREADS, Ld LDH = Ld::Stream, St STH = St::Stream>
 __global__ void __launch_bounds__(THREADS)
@@ -90,6 +96,49 @@ merge_attn_states_lse_kernel(uint16_t *v_out, float *lse_out,
             }
             store<VEC, STH>(v_out + static_cast<int64_t>(v) * VEC, narrow<DT, VEC>(fo));
             if (lse_out != nullptr && v == row[j] * nvec.d) lse_out[row[j]] = mw.lse;
+        }
+    }
+}
+
+}  // namespace astra
+
+namespace astra {
+
+// Same computation for arbitrarily strided tensors (head_dim contiguous): row = token * Hh + head is
+// split again into (token, head) to address each tensor by its own strides.  This is the form for
+// head-major scores ([Hh, T]) or values that are slices of a wider buffer.
+template <int DT, int VEC, int UNROLL, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+merge_attn_states_lse_strided_kernel(uint16_t *v_out, float *lse_out,
+                                     const uint16_t *v_a, const float *lse_a,
+                                     const uint16_t *v_b, const float *lse_b,
+                                     uint32_t total_vecs, uint32_t row0, FastDiv nvec, FastDiv heads,
+                                     MergeStrides st) {
+    const uint32_t base = blockIdx.x * (THREADS * UNROLL) + threadIdx.x;
+    grid_dependency_wait();
+    grid_launch_dependents();
+#pragma unroll
+    for (int j = 0; j < UNROLL; ++j) {
+        const uint32_t v = base + j * THREADS;
+        if (v < total_vecs) {
+            const uint32_t lrow = nvec.div(v);
+            const int64_t col = static_cast<int64_t>(v - lrow * nvec.d) * VEC;
+            const uint32_t row = row0 + lrow;  // rows of this launch start at row0
+            const uint32_t t = heads.div(row);
+            const uint32_t h = row - t * heads.d;
+            const Pack<VEC> a = load<VEC, Ld::Stream>(v_a + (t * st.va_t + h * st.va_h + col));
+            const Pack<VEC> b = load<VEC, Ld::Stream>(v_b + (t * st.vb_t + h * st.vb_h + col));
+            const MergeWeights mw = merge_weights(lse_a[t * st.sa_t + h * st.sa_h], lse_b[t * st.sb_t + h * st.sb_h]);
+            float fa[VEC], fb[VEC], fo[VEC];
+            widen<DT, VEC>(a, fa);
+            widen<DT, VEC>(b, fb);
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                const float ta = mw.use_a ? fa[i] * mw.wa : 0.f;
+                fo[i] = mw.use_b ? fmaf(fb[i], mw.wb, ta) : ta;
+            }
+            store<VEC, St::Stream>(v_out + (t * st.vo_t + h * st.vo_h + col), narrow<DT, VEC>(fo));
+            if (lse_out != nullptr && col == 0) lse_out[t * st.so_t + h * st.so_h] = mw.lse;
         }
     }
 }

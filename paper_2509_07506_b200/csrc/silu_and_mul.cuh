@@ -47,10 +47,13 @@ __device__ __forceinline__ float2 silu_mul2(float2 a, float2 b) {
 
 // Flat indexing: vector v of the output covers out[row, col*VEC .. col*VEC+VEC) with
 // row = v / nvec, col = v % nvec, nvec = D / VEC.  A block handles THREADS*UNROLL consecutive vectors.
+// gate and up are addressed separately (row pitches in elements), which covers both the packed
+// row [a | b] (up = gate + D, equal pitches) and two independent tensors.
 template <int DT, int VEC, int UNROLL, int THREADS, Ld LDH = Ld::StreamReadOnly, St STH = St::Stream>
 __global__ void __launch_bounds__(THREADS)
-silu_and_mul_kernel(uint16_t *__restrict__ out, const uint16_t *__restrict__ in,
-                    uint32_t total_vecs, FastDiv nvec, int64_t D) {
+silu_and_mul_kernel(uint16_t *__restrict__ out, const uint16_t *__restrict__ gate,
+                    const uint16_t *__restrict__ up, uint32_t total_vecs, FastDiv nvec,
+                    int64_t out_pitch, int64_t gate_pitch, int64_t up_pitch) {
     const uint32_t base = blockIdx.x * (THREADS * UNROLL) + threadIdx.x;
     grid_dependency_wait();
     grid_launch_dependents();
@@ -61,9 +64,9 @@ silu_and_mul_kernel(uint16_t *__restrict__ out, const uint16_t *__restrict__ in,
         if (v < total_vecs) {
             const uint32_t row = nvec.div(v);
             const uint32_t col = v - row * nvec.d;
-            const uint16_t *pa = in + (static_cast<int64_t>(row) * 2 * D + static_cast<int64_t>(col) * VEC);
-            a[j] = load<VEC, LDH>(pa);
-            b[j] = load<VEC, LDH>(pa + D);
+            const int64_t c = static_cast<int64_t>(col) * VEC;
+            a[j] = load<VEC, LDH>(gate + (static_cast<int64_t>(row) * gate_pitch + c));
+            b[j] = load<VEC, LDH>(up + (static_cast<int64_t>(row) * up_pitch + c));
         }
     }
 #pragma unroll
@@ -83,7 +86,10 @@ silu_and_mul_kernel(uint16_t *__restrict__ out, const uint16_t *__restrict__ in,
                     fo[i + 1] = o.y;
                 }
             }
-            store<VEC, STH>(out + static_cast<int64_t>(v) * VEC, narrow<DT, VEC>(fo));
+            const uint32_t row = nvec.div(v);
+            const uint32_t col = v - row * nvec.d;
+            store<VEC, STH>(out + (static_cast<int64_t>(row) * out_pitch + static_cast<int64_t>(col) * VEC),
+                            narrow<DT, VEC>(fo));
         }
     }
 }
