@@ -292,6 +292,12 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
         result["shape_sweep"] = shape_sweep(astra, dev, peak)
         result["table4"] = table4_sweep(astra, dev, peak)
         result["strided_variants"] = strided_variants(astra, dev, peak)
+    if world == 1 and not args.no_ablation:
+        from paper_2509_07506_b200 import ablation
+        abl = ablation.run("fp16", dev)
+        result["ablation"] = {"what": "the paper's baseline/optimised design pairs (Section 5.3) rebuilt for sm_100a, "
+                                      "timed beside this library on the Table 4 shapes and the three chain shapes",
+                              "summary": abl["summary"], "rows": abl["rows"], "timing": abl["timing"]}
     if world == 1 and not args.no_cpu:
         result["cpu_baseline"] = oracle_baseline(cfg, rows=min(args.cpu_rows, T))
     return result
@@ -553,6 +559,7 @@ def main() -> int:
     ap.add_argument("--cpu-rows", type=int, default=8192, help="rows of the chain the CPU baseline covers")
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-shape timings of configs[0..3]")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU (oracle) baseline leg")
+    ap.add_argument("--no-ablation", action="store_true", help="skip the design-pair ablation timings")
     ap.add_argument("--no-clocks", action="store_true", help="do not sample clocks with nvidia-smi")
     ap.add_argument("--tokens", type=int, default=wl.CHAIN_T,
                     help="tokens per GPU; the benchmark's workload is the default (8192), smaller values "

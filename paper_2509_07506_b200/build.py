@@ -15,8 +15,10 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB_PATH = os.path.join(PKG_DIR, "libastra.so")
+ABLATION_LIB_PATH = os.path.join(PKG_DIR, "libastra_ablation.so")
 
 SOURCES = ["astra.cu"]
+ABLATION_SOURCES = ["ablation.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
     "-O3", "-std=c++17", "-lineinfo",
@@ -38,26 +40,36 @@ def _inputs():
     return files
 
 
-def is_stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+def is_stale(lib_path: str = LIB_PATH) -> bool:
+    if not os.path.exists(lib_path):
         return True
-    built = os.path.getmtime(LIB_PATH)
+    built = os.path.getmtime(lib_path)
     return any(os.path.getmtime(f) > built for f in _inputs())
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile if the library is missing or older than any source; returns its path."""
-    if not force and not is_stale():
-        return LIB_PATH
-    tmp = LIB_PATH + f".tmp{os.getpid()}"
+def _compile(lib_path: str, sources, force: bool, verbose: bool) -> str:
+    if not force and not is_stale(lib_path):
+        return lib_path
+    tmp = lib_path + f".tmp{os.getpid()}"
     cmd = [_nvcc(), *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += [os.path.join(CSRC, s) for s in SOURCES]
+    cmd += [os.path.join(CSRC, s) for s in sources]
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+    os.replace(tmp, lib_path)
+    return lib_path
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compile libastra.so if it is missing or older than any source; returns its path."""
+    return _compile(LIB_PATH, SOURCES, force, verbose)
+
+
+def build_ablation(force: bool = False, verbose: bool = False) -> str:
+    """Compile libastra_ablation.so (the paper's design pairs, for the ablation measurements)."""
+    return _compile(ABLATION_LIB_PATH, ABLATION_SOURCES, force, verbose)
 
 
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_ablation(force="--force" in sys.argv, verbose="-v" in sys.argv))

@@ -19,24 +19,46 @@ def lib():
     return binding.load_library()
 
 
-def declared_functions():
-    names = set()
-    inc = os.path.join(ROOT, "include")
-    for fn in os.listdir(inc):
-        if fn.endswith(".h"):
-            text = open(os.path.join(inc, fn)).read()
-            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-            names |= set(re.findall(r"\b(astra_[a-z0-9_]+)\s*\(", text))
-    return names
+def declared_functions(header):
+    text = open(os.path.join(ROOT, "include", header)).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return set(re.findall(r"\b(astra_[a-z0-9_]+)\s*\(", text))
 
 
 def test_every_declared_function_is_exported(lib):
-    names = declared_functions()
+    assert sorted(f for f in os.listdir(os.path.join(ROOT, "include")) if f.endswith(".h")) == \
+        ["astra.h", "astra_ablation.h"]
+    names = declared_functions("astra.h")
     assert {"astra_fused_add_rmsnorm", "astra_silu_and_mul", "astra_merge_attn_states_lse",
             "astra_status_string"} <= names
     for n in names:
-        assert hasattr(lib, n), f"{n} is declared in include/ but not exported"
-    assert set(binding.EXPORTED_SYMBOLS) <= names
+        assert hasattr(lib, n), f"{n} is declared in astra.h but not exported by libastra.so"
+    assert set(binding.EXPORTED_SYMBOLS) == names
+
+
+def test_ablation_library_exports_and_argument_errors():
+    from paper_2509_07506_b200 import ablation
+    astra_build.build_ablation()
+    alib = ablation.load_library()
+    names = declared_functions("astra_ablation.h")
+    assert set(ablation.EXPORTED_SYMBOLS) == names
+    for n in names:
+        assert hasattr(alib, n), f"{n} is declared in astra_ablation.h but not exported"
+    f = alib.astra_ablation_fused_add_rmsnorm
+    assert f(0, None, A, A, 1, 8, 1e-6, 0, None) == binding.ASTRA_ERR_NULL_POINTER
+    assert f(2, A, 2 * A, 3 * A, 1, 8, 1e-6, 0, None) == binding.ASTRA_ERR_BAD_SHAPE      # unknown design
+    assert f(1, A, 2 * A, 3 * A, 1, 7, 1e-6, 0, None) == binding.ASTRA_ERR_BAD_SHAPE      # odd width, 32-bit design
+    assert f(1, A + 2, 2 * A, 3 * A, 1, 8, 1e-6, 0, None) == binding.ASTRA_ERR_MISALIGNED
+    assert f(0, A, 2 * A, 3 * A, 0, 8, 1e-6, 0, None) == binding.ASTRA_OK
+    g = alib.astra_ablation_silu_and_mul
+    assert g(0, A, None, 1, 8, 0, None) == binding.ASTRA_ERR_NULL_POINTER
+    assert g(1, A, 2 * A, 1, 9, 0, None) == binding.ASTRA_ERR_BAD_SHAPE
+    assert g(0, A, 2 * A, 1, 8, 4, None) == binding.ASTRA_ERR_BAD_DTYPE
+    assert g(1, A, 2 * A, 0, 8, 0, None) == binding.ASTRA_OK
+    h = alib.astra_ablation_merge_attn_states_lse
+    assert h(0, A, None, A, A, A, A, 1, 1, 8, 0, None) == binding.ASTRA_ERR_NULL_POINTER
+    assert h(1, A, A, A, A, A, A, 1, 1, 9, 0, None) == binding.ASTRA_ERR_BAD_SHAPE
+    assert h(0, A, A, A, A, A, A, 0, 1, 8, 0, None) == binding.ASTRA_OK
 
 
 def test_status_strings(lib):
