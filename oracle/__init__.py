@@ -26,40 +26,51 @@ _LIB = os.path.join(_HERE, "liboracle.so")
 _lib = None
 
 
+def compile_source(src: str, out: str) -> str:
+    """gcc command used for the oracle (no fast-math, no contraction)."""
+    subprocess.check_call(
+        ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared",
+         "-ffp-contract=off", "-fno-fast-math", "-o", out, src, "-lm"]
+    )
+    return out
+
+
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc; returns the path of the shared object."""
     stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
     if force or stale:
         tmp = _LIB + f".tmp{os.getpid()}"
-        subprocess.check_call(
-            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared",
-             "-ffp-contract=off", "-fno-fast-math", "-o", tmp, _SRC, "-lm"]
-        )
+        compile_source(_SRC, tmp)
         os.replace(tmp, _LIB)
     return _LIB
+
+
+def declare(lib):
+    """Attach the C prototypes to a loaded oracle library (also used by the tests that load
+    deliberately broken copies of the source)."""
+    u16p = ctypes.POINTER(ctypes.c_uint16)
+    f32p = ctypes.POINTER(ctypes.c_float)
+    f64p = ctypes.POINTER(ctypes.c_double)
+    i64 = ctypes.c_int64
+    lib.oracle_widen.argtypes = [ctypes.c_uint16, ctypes.c_int]
+    lib.oracle_widen.restype = ctypes.c_double
+    lib.oracle_round_to_storage.argtypes = [ctypes.c_double, ctypes.c_int]
+    lib.oracle_round_to_storage.restype = ctypes.c_uint16
+    lib.oracle_fused_add_rmsnorm.argtypes = [u16p, u16p, u16p, i64, i64, ctypes.c_float,
+                                             ctypes.c_int, f64p, u16p, ctypes.c_int]
+    lib.oracle_fused_add_rmsnorm.restype = None
+    lib.oracle_silu_and_mul.argtypes = [u16p, i64, i64, ctypes.c_int, f64p, ctypes.c_int]
+    lib.oracle_silu_and_mul.restype = None
+    lib.oracle_merge_attn_states_lse.argtypes = [u16p, f32p, u16p, f32p, i64, i64, i64,
+                                                 ctypes.c_int, f64p, f64p, ctypes.c_int]
+    lib.oracle_merge_attn_states_lse.restype = None
+    return lib
 
 
 def _load():
     global _lib
     if _lib is None:
-        lib = ctypes.CDLL(build())
-        u16p = ctypes.POINTER(ctypes.c_uint16)
-        f32p = ctypes.POINTER(ctypes.c_float)
-        f64p = ctypes.POINTER(ctypes.c_double)
-        i64 = ctypes.c_int64
-        lib.oracle_widen.argtypes = [ctypes.c_uint16, ctypes.c_int]
-        lib.oracle_widen.restype = ctypes.c_double
-        lib.oracle_round_to_storage.argtypes = [ctypes.c_double, ctypes.c_int]
-        lib.oracle_round_to_storage.restype = ctypes.c_uint16
-        lib.oracle_fused_add_rmsnorm.argtypes = [u16p, u16p, u16p, i64, i64, ctypes.c_float,
-                                                 ctypes.c_int, f64p, u16p, ctypes.c_int]
-        lib.oracle_fused_add_rmsnorm.restype = None
-        lib.oracle_silu_and_mul.argtypes = [u16p, i64, i64, ctypes.c_int, f64p, ctypes.c_int]
-        lib.oracle_silu_and_mul.restype = None
-        lib.oracle_merge_attn_states_lse.argtypes = [u16p, f32p, u16p, f32p, i64, i64, i64,
-                                                     ctypes.c_int, f64p, f64p, ctypes.c_int]
-        lib.oracle_merge_attn_states_lse.restype = None
-        _lib = lib
+        _lib = declare(ctypes.CDLL(build()))
     return _lib
 
 

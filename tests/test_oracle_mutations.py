@@ -1,0 +1,117 @@
+"""Do the pins bite?  Each case plants one plausible mistake in a COPY of the oracle's C source
+(a dropped term, a wrong sign, a swapped operand, a misplaced epsilon, ...), builds it on the CPU,
+swaps it in for the real oracle, and requires that at least one pin in test_oracle_pins.py fails.
+A mistake that no pin catches would mean the oracle is not pinned against it."""
+import ctypes
+import inspect
+import os
+
+import pytest
+
+import oracle
+import test_oracle_pins as pins
+
+SRC = os.path.join(os.path.dirname(os.path.abspath(oracle.__file__)), "astra_oracle.c")
+
+# (name, text in the oracle source, replacement)
+MUTATIONS = [
+    ("rmsnorm: eps added outside the root",
+     "sqrt(sum_sq / (double)H + (double)eps)", "(sqrt(sum_sq / (double)H) + (double)eps)"),
+    ("rmsnorm: sum of squares instead of mean",
+     "sqrt(sum_sq / (double)H + (double)eps)", "sqrt(sum_sq + (double)eps)"),
+    ("rmsnorm: eps dropped",
+     "sqrt(sum_sq / (double)H + (double)eps)", "sqrt(sum_sq / (double)H)"),
+    ("rmsnorm: weight indexed from the other end",
+     "/ denom * widen(w[j], f)", "/ denom * widen(w[H - 1 - j], f)"),
+    ("rmsnorm: weight dropped",
+     "/ denom * widen(w[j], f)", "/ denom"),
+    ("rmsnorm: norm taken from the stored residual instead of the binary32 sum",
+     "double s = (double)(float)s_exact;                  /* binary32 add    */",
+     "double s = widen(round_to_storage((double)(float)s_exact, f), f);"),
+    ("rmsnorm: x - r instead of x + r (both loops)",
+     "widen(xt[j], f) + widen(rt[j], f)", "widen(xt[j], f) - widen(rt[j], f)"),
+    ("rmsnorm: residual gets x only",
+     "float s32 = (float)s_exact;", "float s32 = (float)widen(xt[j], f);"),
+    ("rmsnorm: divides by the mean square instead of its root",
+     "double denom = sqrt(", "double denom = ("),
+    ("silu: e^{+z} in the denominator",
+     "return z / (1.0 + exp(-z));", "return z / (1.0 + exp(z));"),
+    ("silu: sigmoid instead of SiLU (z dropped)",
+     "return z / (1.0 + exp(-z));", "return 1.0 / (1.0 + exp(-z));"),
+    ("silu: gate and up halves swapped",
+     "double a = widen(row[i], f);\n            double b = widen(row[D + i], f);",
+     "double a = widen(row[D + i], f);\n            double b = widen(row[i], f);"),
+    ("silu: multiplication by b dropped",
+     "out[t * D + i] = silu(a) * b;", "out[t * D + i] = silu(a);"),
+    ("silu: row pitch D instead of 2D",
+     "const uint16_t *row = input + t * 2 * D;", "const uint16_t *row = input + t * D;"),
+    ("merge: weights applied to the wrong states",
+     "if (wa != 0.0) num += wa * widen(va[d], f);\n            if (wb != 0.0) num += wb * widen(vb[d], f);",
+     "if (wa != 0.0) num += wa * widen(vb[d], f);\n            if (wb != 0.0) num += wb * widen(va[d], f);"),
+    ("merge: normalisation dropped",
+     "vo[d] = num / denom;", "vo[d] = num;"),
+    ("merge: max dropped from the merged score",
+     "lse_out[th] = m + log(denom);", "lse_out[th] = log(denom);"),
+    ("merge: score is log of the max weight only",
+     "lse_out[th] = m + log(denom);", "lse_out[th] = m;"),
+    ("merge: difference of scores with the wrong sign",
+     "double wa = exp(sa - m);", "double wa = exp(m - sa);"),
+    ("merge: both-empty case not handled",
+     "if (sa == -INFINITY && sb == -INFINITY) {", "if (0) {"),
+    ("merge: zero-weight side multiplied instead of skipped",
+     "if (wb != 0.0) num += wb * widen(vb[d], f);", "num += wb * widen(vb[d], f);"),
+    ("merge: scores indexed per token instead of per (token, head)",
+     "double sb = (double)lse_b[th];", "double sb = (double)lse_b[th / Hh];"),
+    ("storage: fp16 exponent bias off by one",
+     "f.frac_bits = 10; f.exp_bits = 5; f.bias = 15;", "f.frac_bits = 10; f.exp_bits = 5; f.bias = 16;"),
+    ("storage: bf16 read with 8 fraction bits",
+     "f.frac_bits = 7;  f.exp_bits = 8; f.bias = 127;", "f.frac_bits = 8;  f.exp_bits = 8; f.bias = 127;"),
+    ("storage: truncation instead of round-to-nearest-even",
+     "double q = nearbyint(a / quantum);", "double q = floor(a / quantum);"),
+    ("storage: round half away from zero",
+     "double q = nearbyint(a / quantum);", "double q = floor(a / quantum + 0.5);"),
+    ("storage: subnormals flushed on widening",
+     "v = ldexp((double)frac, 1 - f.bias - f.frac_bits);", "v = 0.0;"),
+]
+
+PIN_TESTS = [(name, fn) for name, fn in inspect.getmembers(pins, inspect.isfunction) if name.startswith("test_")]
+
+
+def run_all_pins():
+    """Calls every pin with every parameter combination; returns the names of those that failed."""
+    failed = []
+    for name, fn in PIN_TESTS:
+        marks = [m for m in getattr(fn, "pytestmark", []) if m.name == "parametrize"]
+        combos = [{}]
+        for m in marks:
+            argnames = [a.strip() for a in m.args[0].split(",")]
+            new = []
+            for c in combos:
+                for vals in m.args[1]:
+                    vals = vals if isinstance(vals, (tuple, list)) and len(argnames) > 1 else (vals,)
+                    d = dict(c); d.update(dict(zip(argnames, vals)))
+                    new.append(d)
+            combos = new
+        for kw in combos:
+            try:
+                fn(**kw)
+            except Exception:  # an assertion, or an arithmetic error caused by the planted mistake
+                failed.append(name)
+                break
+    return failed
+
+
+def test_unmodified_oracle_passes_when_driven_this_way():
+    assert run_all_pins() == []
+
+
+@pytest.mark.parametrize("name,old,new", MUTATIONS, ids=[m[0] for m in MUTATIONS])
+def test_planted_mistake_is_caught(name, old, new, tmp_path, monkeypatch):
+    text = open(SRC).read()
+    assert text.count(old) >= 1, f"mutation target not found in the oracle source: {old!r}"
+    src = tmp_path / "mutated.c"
+    src.write_text(text.replace(old, new))
+    lib = oracle.declare(ctypes.CDLL(oracle.compile_source(str(src), str(tmp_path / "libmutated.so"))))
+    monkeypatch.setattr(oracle, "_lib", lib)
+    failed = run_all_pins()
+    assert failed, f"no pin noticed: {name}"

@@ -391,6 +391,8 @@ def test_merge_neg_inf_returns_other_state(dtype):
     # a non-finite payload on the zero-weight side does not leak
     v, s = _merge([[[float("inf"), float("nan"), 1.0, 1.0]]], [[ninf]], vb, [[0.5]], dtype)
     assert np.array_equal(v[0, 0], np.array(vb[0][0])) and s[0, 0] == 0.5
+    v, s = _merge(va, [[-2.5]], [[[float("nan"), float("-inf"), 1.0, 1.0]]], [[ninf]], dtype)
+    assert np.array_equal(v[0, 0], np.array(va[0][0])) and s[0, 0] == -2.5
 
 
 def test_merge_out_of_domain_scores_give_nan():
