@@ -6,8 +6,8 @@
 // thread block owns one row.  In the register-resident kernel each thread keeps its share of the
 // binary32 sums s in registers across the row reduction, so the row makes a single trip through
 // HBM.  The reduction is the one the paper's optimised kernel uses: shuffles inside each warp, one
-// shared-memory slot per warp, then a short combine.  All loads of a row (x, r and w) are issued
-// before anything is consumed.
+// shared-memory slot per warp, then a short combine.  All loads of x and r of a row are issued
+// before anything is consumed; the weight (an L2 hit) is fetched while the reduction completes.
 #pragma once
 
 #include "vec.cuh"
@@ -49,8 +49,14 @@ __host__ __device__ constexpr int rmsnorm_reg_max_threads(int vec, int vpt) {
 
 // Register-resident row: thread i owns vectors i, i + blockDim.x, ... (at most VPT of them).
 // Requires nvec = H / VEC <= VPT * blockDim.x and blockDim.x <= rmsnorm_reg_max_threads(VEC, VPT).
-template <int DT, int VEC, int VPT, Ld LDH = Ld::Stream, St STH = St::Stream>
-__global__ void __launch_bounds__(rmsnorm_reg_max_threads(VEC, VPT))
+// EARLY_W issues the weight loads before the reduction instead of after it (measured: no faster,
+// and it costs the registers that decide occupancy).  MINB is the minimum number of resident blocks
+// the register allocation must allow; with 16 elements per thread MINB = 2 caps the kernel at 32
+// registers, i.e. full occupancy for every block size, which is worth 5 % at [16384, 8192] and
+// 27 % at [512, 14336] (896-thread blocks: two per SM instead of one).
+template <int DT, int VEC, int VPT, Ld LDH = Ld::Stream, St STH = St::Stream, bool EARLY_W = false,
+          int MINB = (VEC * VPT <= 16 ? 2 : 1)>
+__global__ void __launch_bounds__(rmsnorm_reg_max_threads(VEC, VPT), MINB)
 fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ weight,
                              int H, float eps, float inv_H) {
     __shared__ float slots[kMaxWarps];
@@ -73,10 +79,12 @@ fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ we
             pr[i] = load<VEC, LDH>(rr + v * VEC);
         }
     }
+    if constexpr (EARLY_W) {
 #pragma unroll
-    for (int i = 0; i < VPT; ++i) {
-        const int v = threadIdx.x + i * blockDim.x;
-        if (v < nvec) pw[i] = load<VEC, Ld::Keep>(weight + v * VEC);
+        for (int i = 0; i < VPT; ++i) {
+            const int v = threadIdx.x + i * blockDim.x;
+            if (v < nvec) pw[i] = load<VEC, Ld::Keep>(weight + v * VEC);
+        }
     }
 
     float s[VPT][VEC];
@@ -97,6 +105,13 @@ fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ we
         }
     }
 
+    if constexpr (!EARLY_W) {
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int v = threadIdx.x + i * blockDim.x;
+            if (v < nvec) pw[i] = load<VEC, Ld::Keep>(weight + v * VEC);
+        }
+    }
     const float total = block_sum(acc, slots);
     const float rstd = rsqrtf(fmaf(total, inv_H, eps));
 
