@@ -316,3 +316,26 @@ def test_binding_rejects_wrong_arguments():
     with pytest.raises(astra.AstraError) as e:
         astra.astra_fused_add_rmsnorm(x, x, x[0].clone(), 1e-6)
     assert e.value.status == 6
+
+
+def test_host_streamer_pipeline_matches_oracle():
+    """Host-resident batches processed in row chunks over three streams, device buffers reused
+    for a second batch: results of both batches match the oracle."""
+    from paper_2509_07506_b200.hoststream import HostStreamer
+    dev = torch.device("cuda", torch.cuda.current_device())
+    T, D, chunk = 96, 1000, 32
+    pipe = HostStreamer(dev)
+    d_in = torch.empty((T, 2 * D), dtype=torch.bfloat16, device=dev)
+    d_out = torch.empty((T, D), dtype=torch.bfloat16, device=dev)
+    batches = [wl.silu_inputs(T, D, BF16, seed=s) for s in (41, 42)]
+    host_in = [b.input.pin_memory() for b in batches]
+    host_out = [torch.empty((T, D), dtype=torch.bfloat16).pin_memory() for _ in batches]
+    for hin, hout in zip(host_in, host_out):
+        for r0 in range(0, T, chunk):
+            sl = slice(r0, r0 + chunk)
+            pipe.submit(("silu", r0), [(d_in[sl], hin[sl])],
+                        lambda sl=sl: astra.astra_silu_and_mul(d_out[sl], d_in[sl]),
+                        [(hout[sl], d_out[sl])])
+    pipe.synchronize()
+    for b, hout in zip(batches, host_out):
+        check_values(f64(hout), oracle.silu_and_mul(wl.bits(b.input), BF16), BF16, what="host streamer")
