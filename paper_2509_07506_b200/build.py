@@ -47,11 +47,11 @@ def is_stale(lib_path: str = LIB_PATH) -> bool:
     return any(os.path.getmtime(f) > built for f in _inputs())
 
 
-def _compile(lib_path: str, sources, force: bool, verbose: bool) -> str:
+def _compile(lib_path: str, sources, force: bool, verbose: bool, extra_flags=()) -> str:
     if not force and not is_stale(lib_path):
         return lib_path
     tmp = lib_path + f".tmp{os.getpid()}"
-    cmd = [_nvcc(), *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-o", tmp]
+    cmd = [_nvcc(), *NVCC_FLAGS, *extra_flags, "-I", INCLUDE, "-I", CSRC, "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in sources]
@@ -63,6 +63,13 @@ def _compile(lib_path: str, sources, force: bool, verbose: bool) -> str:
 def build(force: bool = False, verbose: bool = False) -> str:
     """Compile libastra.so if it is missing or older than any source; returns its path."""
     return _compile(LIB_PATH, SOURCES, force, verbose)
+
+
+def build_variant(lib_path: str, defines: dict) -> str:
+    """Compile libastra's sources to `lib_path` with extra preprocessor definitions (used by the
+    tests to lower the per-launch limits so that the multi-launch splitting runs on small inputs)."""
+    flags = [f"-D{k}={v}" for k, v in defines.items()]
+    return _compile(lib_path, SOURCES, True, False, flags)
 
 
 def build_ablation(force: bool = False, verbose: bool = False) -> str:

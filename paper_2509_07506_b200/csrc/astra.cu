@@ -83,7 +83,16 @@ inline void launch(void (*kernel)(KArgs...), unsigned grid, unsigned block, cuda
     (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);  // failure is read back by launch_status()
 }
 
-constexpr int64_t kMaxVecsPerLaunch = (1ll << 31) - 1;  // flat vector indices are 31-bit
+// Flat vector indices are 31-bit and grids are limited to 2^31-1 blocks; larger inputs are split
+// into several launches.  The two limits can be lowered at compile time so that tests can drive the
+// splitting with small inputs.
+#ifndef ASTRA_MAX_VECS_PER_LAUNCH
+#define ASTRA_MAX_VECS_PER_LAUNCH ((1ll << 31) - 1)
+#endif
+#ifndef ASTRA_MAX_ROWS_PER_LAUNCH
+#define ASTRA_MAX_ROWS_PER_LAUNCH 2147483647
+#endif
+constexpr int64_t kMaxVecsPerLaunch = ASTRA_MAX_VECS_PER_LAUNCH;
 constexpr int64_t kInt64Max = 9223372036854775807ll;
 
 inline bool valid_dtype(astra_dtype_t d) { return d == ASTRA_BF16 || d == ASTRA_FP16; }
@@ -235,7 +244,7 @@ inline bool rows_disjoint(int64_t T, int64_t Hh, int64_t W, int64_t st, int64_t 
 // ---------------------------------------------------------------------------------------------
 // fused_add_rmsnorm
 // ---------------------------------------------------------------------------------------------
-constexpr int kMaxGridX = 2147483647;
+constexpr int kMaxGridX = ASTRA_MAX_ROWS_PER_LAUNCH;
 
 // Most elements of a row one thread keeps in registers: 64 with vector accesses, 16 on the scalar
 // path (each element then also costs three separate packed-input registers).
