@@ -155,7 +155,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
     import paper_2509_07506_b200 as astra
     import torch.distributed as dist
 
-    dev = torch.device("cuda", local_rank)
+    dev = torch.device("cuda", local_rank % torch.cuda.device_count())
     torch.cuda.set_device(dev)
     astra.load_library()  # fails loudly if the CUDA library is missing
     T = args.tokens
@@ -174,7 +174,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local_rank) if (rank == 0 and not args.no_clocks) else None
+    sampler = ClockSampler(dev.index) if (rank == 0 and not args.no_clocks) else None
     K, W = args.steps, args.warmup
     for _ in range(W):
         step()
@@ -273,7 +273,8 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
     e2e_ms = e0.elapsed_time(e1)
 
     # ---- max over ranks -------------------------------------------------------------------------
-    times = multi.max_over_ranks([total_ms, e2e_ms] + [kernel_ms[n] for n in names], device=dev)
+    times = multi.max_over_ranks([total_ms, e2e_ms] + [kernel_ms[n] for n in names],
+                                 device=dev if args.backend == "nccl" else "cpu")
     total_ms, e2e_ms = float(times[0]), float(times[1])
     kernel_ms = {n: float(times[2 + j]) for j, n in enumerate(names)}
 
@@ -592,6 +593,9 @@ def main() -> int:
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU (oracle) baseline leg")
     ap.add_argument("--no-ablation", action="store_true", help="skip the design-pair ablation timings")
     ap.add_argument("--no-clocks", action="store_true", help="do not sample clocks with nvidia-smi")
+    ap.add_argument("--backend", choices=["nccl", "gloo"], default="nccl",
+                    help="process-group backend for the timing reduction when WORLD_SIZE > 1 (gloo allows a "
+                         "functional check of the multi-rank path with several ranks sharing one GPU)")
     ap.add_argument("--tokens", type=int, default=wl.CHAIN_T,
                     help="tokens per GPU; the benchmark's workload is the default (8192), smaller values "
                          "are for profiler captures")
@@ -611,7 +615,7 @@ def main() -> int:
         print("bench.py: no CUDA device; the CUDA library has no CPU fallback", file=sys.stderr)
         return 1
     if world > 1:
-        multi.init_process_group("nccl", torch.device("cuda", local_rank))
+        multi.init_process_group(args.backend, torch.device("cuda", local_rank % torch.cuda.device_count()))
     try:
         res = run_astra(args, rank, world, local_rank)
     finally:
