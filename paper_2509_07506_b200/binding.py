@@ -100,9 +100,17 @@ def _code(t: torch.Tensor, name: str) -> int:
     return _DTYPE_CODE[t.dtype]
 
 
+# torch's C accessor for the current stream handle; about 2 us cheaper per call than building a
+# torch.cuda.Stream object just to read its handle.
+_raw_current_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
 def _stream(t: torch.Tensor, stream: Optional[torch.cuda.Stream]) -> int:
-    s = stream if stream is not None else torch.cuda.current_stream(t.device)
-    return s.cuda_stream
+    if stream is not None:
+        return stream.cuda_stream
+    if _raw_current_stream is not None:
+        return _raw_current_stream(t.device.index)
+    return torch.cuda.current_stream(t.device).cuda_stream
 
 
 class _on_device:
