@@ -25,3 +25,14 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """Compile the CUDA libraries and the C oracle if they are missing or older than their sources
+    (nvcc and gcc need no GPU), so that a fresh checkout can run either half of the suite."""
+    from paper_2509_07506_b200 import build as astra_build
+    astra_build.build()
+    astra_build.build_ablation()
+    import oracle
+    oracle.build()
