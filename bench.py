@@ -329,6 +329,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
         result["shape_sweep"] = shape_sweep(astra, dev, peak)
         result["table4"] = table4_sweep(astra, dev, peak)
         result["strided_variants"] = strided_variants(astra, dev, peak)
+        result["decode_chain"] = decode_chain(astra, dev)
     if world == 1 and not args.no_ablation:
         from paper_2509_07506_b200 import ablation
         astra_build.build_ablation()
@@ -446,6 +447,33 @@ def shape_sweep(astra, dev, peak) -> list:
         for T in wl.SWEEP_T:
             for H in wl.SWEEP_H:
                 rms(dtype, T, H)
+    return rows
+
+
+def decode_chain(astra, dev) -> list:
+    """The three-call chain at decode-sized token counts (launch-latency bound): us per chain step
+    through the binding call by call, and replayed from a CUDA graph of 20 steps (device time; the
+    kernels' dependent-launch hooks let each launch overlap the previous kernel's drain)."""
+    rows = []
+    bf = torch.bfloat16
+    H, D, Hh, Dh = wl.CHAIN_H, wl.CHAIN_D, wl.CHAIN_HEADS, wl.CHAIN_HEAD_DIM
+    for T in (1, 16, 64, 256):
+        x = torch.randn((T, H), device=dev).to(bf); r = torch.randn((T, H), device=dev).to(bf)
+        w = torch.ones((H,), device=dev, dtype=bf)
+        si = torch.randn((T, 2 * D), device=dev).to(bf); so = torch.empty((T, D), device=dev, dtype=bf)
+        va = torch.randn((T, Hh, Dh), device=dev).to(bf); vb = torch.randn((T, Hh, Dh), device=dev).to(bf)
+        vo = torch.empty_like(va)
+        sa = torch.rand((T, Hh), device=dev) * 30 - 10; sb = torch.rand((T, Hh), device=dev) * 30 - 10
+        lo = torch.empty_like(sa)
+
+        def step(_=None):
+            astra.astra_fused_add_rmsnorm(x, r, w, 1e-5)
+            astra.astra_silu_and_mul(so, si)
+            astra.astra_merge_attn_states_lse(vo, lo, va, sa, vb, sb)
+
+        eager = _time_launches(step)
+        graph = _time_graph(step, [None], launches=20)
+        rows.append({"tokens": T, "us_per_step_eager": round(eager, 2), "us_per_step_graph": round(graph, 2)})
     return rows
 
 
