@@ -330,6 +330,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
         result["table4"] = table4_sweep(astra, dev, peak)
         result["strided_variants"] = strided_variants(astra, dev, peak)
         result["decode_chain"] = decode_chain(astra, dev)
+        result["fp32_variants"] = fp32_variants(astra, dev, peak)
     if world == 1 and not args.no_ablation:
         from paper_2509_07506_b200 import ablation
         astra_build.build_ablation()
@@ -510,6 +511,32 @@ def strided_variants(astra, dev, peak) -> list:
     so = torch.empty((Hh, T), device=dev).t()
     add("astra_merge_attn_states_lse_ex head-major scores [8192,32,128]", wl.merge_bytes(T, Hh, Dh),
         lambda: astra.astra_merge_attn_states_lse_ex(vo, so, va, sa, vb, sb))
+    return rows
+
+
+def fp32_variants(astra, dev, peak) -> list:
+    """The three operations on fp32 storage at the chain shapes (twice the bytes of the bf16 calls)."""
+    T, H, D, Hh, Dh = wl.CHAIN_T, wl.CHAIN_H, wl.CHAIN_D, wl.CHAIN_HEADS, wl.CHAIN_HEAD_DIM
+    rows = []
+
+    def add(name, nbytes, fn):
+        us = _time_launches(fn)
+        gbs = nbytes / (us * 1e-6) / 1e9
+        rows.append({"call": name, "us_per_call": round(us, 2), "gbs": round(gbs, 1),
+                     "frac_of_measured_peak": round(gbs / peak, 4)})
+
+    x = torch.randn((T, H), device=dev); r = torch.randn((T, H), device=dev); w = torch.ones((H,), device=dev)
+    add("astra_fused_add_rmsnorm fp32 [8192,4096]", wl.rmsnorm_bytes(T, H, 4),
+        lambda: astra.astra_fused_add_rmsnorm(x, r, w, 1e-5))
+    del x, r, w
+    si = torch.randn((T, 2 * D), device=dev); so = torch.empty((T, D), device=dev)
+    add("astra_silu_and_mul fp32 [8192,2*14336]", wl.silu_bytes(T, D, 4), lambda: astra.astra_silu_and_mul(so, si))
+    del si, so
+    va = torch.randn((T, Hh, Dh), device=dev); vb = torch.randn((T, Hh, Dh), device=dev); vo = torch.empty_like(va)
+    sa = torch.rand((T, Hh), device=dev) * 30 - 10; sb = torch.rand((T, Hh), device=dev) * 30 - 10
+    lo = torch.empty_like(sa)
+    add("astra_merge_attn_states_lse fp32 [8192,32,128]", wl.merge_bytes(T, Hh, Dh, 4),
+        lambda: astra.astra_merge_attn_states_lse(vo, lo, va, sa, vb, sb))
     return rows
 
 

@@ -9,10 +9,11 @@
  *     work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream)
  *     and the call returns immediately.  Host pointers are not detected (undefined behaviour).
  *   - Tensors are dense and row-major (the last index is contiguous; a row's pitch is its width).
- *   - `dtype` selects the 16-bit storage type of all value tensors of the call.  Arithmetic is
- *     binary32 throughout, with a single round-to-nearest-even to the storage type at each store.
- *   - Pointers need only the natural alignment of their element (2 bytes for values, 4 for
- *     scores).  Wider alignment is detected and exploited inside; widths need not be multiples
+ *   - `dtype` selects the storage type of all value tensors of the call (bf16, fp16 or fp32).
+ *     Arithmetic is binary32 throughout, with a single round-to-nearest-even to the storage type at
+ *     each store.
+ *   - Pointers need only the natural alignment of their element (2 bytes for 16-bit values, 4 for
+ *     fp32 values and for scores).  Wider alignment is detected and exploited inside; widths need not be multiples
  *     of 8.  A pointer with less than element alignment gives ASTRA_ERR_MISALIGNED.
  *   - Errors are return codes only: nothing is printed, thrown or aborted, and on any error
  *     nothing has been launched.  A zero-sized first dimension (T == 0) is ASTRA_OK and launches
@@ -30,7 +31,8 @@ extern "C" {
 
 typedef enum {
     ASTRA_BF16 = 0, /* bfloat16: 1 sign, 8 exponent, 7 fraction bits */
-    ASTRA_FP16 = 1  /* IEEE binary16                                  */
+    ASTRA_FP16 = 1, /* IEEE binary16                                  */
+    ASTRA_FP32 = 2  /* IEEE binary32 (no conversion, no rounding at the store beyond the arithmetic's own) */
 } astra_dtype_t;
 
 typedef enum {

@@ -6,7 +6,7 @@ Only the tests, the smoke check and the CPU-baseline leg of the benchmark may
 import this package; the CUDA library and its Python binding never do, and this
 package imports nothing from them.
 
-Arrays are numpy: 16-bit storage patterns as ``uint16``, scores as ``float32``,
+Arrays are numpy: storage patterns as ``uint16`` (bf16, fp16) or ``uint32`` (fp32), scores as ``float32``,
 results as ``float64`` (and ``uint16`` for the bit-exact residual).
 """
 from __future__ import annotations
@@ -19,6 +19,7 @@ import numpy as np
 
 BF16 = 0
 FP16 = 1
+FP32 = 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "astra_oracle.c")
@@ -48,7 +49,7 @@ def build(force: bool = False) -> str:
 def declare(lib):
     """Attach the C prototypes to a loaded oracle library (also used by the tests that load
     deliberately broken copies of the source)."""
-    u16p = ctypes.POINTER(ctypes.c_uint16)
+    u16p = ctypes.c_void_p  # value tensors: uint16 patterns (bf16, fp16) or uint32 patterns (fp32)
     f32p = ctypes.POINTER(ctypes.c_float)
     f64p = ctypes.POINTER(ctypes.c_double)
     i64 = ctypes.c_int64
@@ -74,10 +75,12 @@ def _load():
     return _lib
 
 
-def _u16(a, shape):
+def _u16(a, shape, dtype=BF16):
+    """Storage patterns of a value tensor: uint16 for the 16-bit types, uint32 for fp32."""
     a = np.ascontiguousarray(a)
-    if a.dtype != np.uint16:
-        raise TypeError(f"expected uint16 storage patterns, got {a.dtype}")
+    want = np.uint32 if dtype == FP32 else np.uint16
+    if a.dtype != want:
+        raise TypeError(f"expected {np.dtype(want).name} storage patterns, got {a.dtype}")
     if tuple(a.shape) != tuple(shape):
         raise ValueError(f"expected shape {tuple(shape)}, got {tuple(a.shape)}")
     return a
@@ -93,6 +96,8 @@ def _f32(a, shape):
 
 
 def _ptr(a, ctype):
+    if ctype is ctypes.c_uint16:  # value tensor: passed as void*
+        return ctypes.c_void_p(a.ctypes.data)
     return a.ctypes.data_as(ctypes.POINTER(ctype))
 
 
@@ -107,14 +112,14 @@ def round_to_storage(value: float, dtype: int) -> int:
 
 
 def fused_add_rmsnorm(x, residual, weight, eps: float, dtype: int, nthreads: int = 1):
-    """Table 1, Kernel 2.  Returns (y float64 [T,H], residual_out uint16 [T,H])."""
+    """Table 1, Kernel 2.  Returns (y float64 [T,H], residual_out storage patterns [T,H])."""
     x = np.ascontiguousarray(x)
     T, H = x.shape
-    x = _u16(x, (T, H))
-    residual = _u16(residual, (T, H))
-    weight = _u16(weight, (H,))
+    x = _u16(x, (T, H), dtype)
+    residual = _u16(residual, (T, H), dtype)
+    weight = _u16(weight, (H,), dtype)
     y = np.empty((T, H), dtype=np.float64)
-    r_out = np.empty((T, H), dtype=np.uint16)
+    r_out = np.empty((T, H), dtype=x.dtype)
     _load().oracle_fused_add_rmsnorm(
         _ptr(x, ctypes.c_uint16), _ptr(residual, ctypes.c_uint16), _ptr(weight, ctypes.c_uint16),
         T, H, np.float32(eps).item(), int(dtype),
@@ -129,7 +134,7 @@ def silu_and_mul(inp, dtype: int, nthreads: int = 1):
     if twoD % 2:
         raise ValueError("last dimension must be even")
     D = twoD // 2
-    inp = _u16(inp, (T, twoD))
+    inp = _u16(inp, (T, twoD), dtype)
     out = np.empty((T, D), dtype=np.float64)
     _load().oracle_silu_and_mul(_ptr(inp, ctypes.c_uint16), T, D, int(dtype),
                                 _ptr(out, ctypes.c_double), int(nthreads))
@@ -140,8 +145,8 @@ def merge_attn_states_lse(v_a, lse_a, v_b, lse_b, dtype: int, nthreads: int = 1)
     """Table 1, Kernel 1.  Returns (v_out float64 [T,Hh,D], lse_out float64 [T,Hh])."""
     v_a = np.ascontiguousarray(v_a)
     T, Hh, D = v_a.shape
-    v_a = _u16(v_a, (T, Hh, D))
-    v_b = _u16(v_b, (T, Hh, D))
+    v_a = _u16(v_a, (T, Hh, D), dtype)
+    v_b = _u16(v_b, (T, Hh, D), dtype)
     lse_a = _f32(lse_a, (T, Hh))
     lse_b = _f32(lse_b, (T, Hh))
     v_out = np.empty((T, Hh, D), dtype=np.float64)

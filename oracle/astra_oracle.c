@@ -14,7 +14,9 @@
  * arithmetic because rows never interact.
  *
  * Storage formats.  dtype 0 = bfloat16 (1 sign, 8 exponent, 7 fraction bits),
- * dtype 1 = IEEE binary16 (1, 5, 10).  Both are widened exactly to double and
+ * dtype 1 = IEEE binary16 (1, 5, 10), dtype 2 = IEEE binary32 (value tensors are
+ * then arrays of 32-bit patterns; the C compiler's float is that format, so it is
+ * widened by a cast and rounded by a cast).  The 16-bit formats are widened exactly to double and
  * rounded back with round-to-nearest-even, written out arithmetically below
  * (frexp / ldexp / nearbyint), not with bit tricks, so they can be read against
  * the format definitions.
@@ -31,6 +33,7 @@
 
 #define ORACLE_BF16 0
 #define ORACLE_FP16 1
+#define ORACLE_FP32 2 /* IEEE binary32 storage: patterns are 32 bits wide */
 
 typedef struct {
     int frac_bits; /* explicit fraction bits            */
@@ -43,7 +46,7 @@ static storage_format format_of(int dtype)
     storage_format f;
     if (dtype == ORACLE_FP16) {
         f.frac_bits = 10; f.exp_bits = 5; f.bias = 15;
-    } else {
+    } else { /* bfloat16; binary32 storage never goes through this table */
         f.frac_bits = 7;  f.exp_bits = 8; f.bias = 127;
     }
     return f;
@@ -118,6 +121,27 @@ uint16_t oracle_round_to_storage(double v, int dtype)
     return round_to_storage(v, format_of(dtype));
 }
 
+/* Element i of a value tensor of the given storage type, as its exact double value. */
+static double load_value(const void *base, int64_t i, int dtype, storage_format f)
+{
+    if (dtype == ORACLE_FP32) {
+        float v;
+        memcpy(&v, (const unsigned char *)base + 4 * i, 4);
+        return (double)v;
+    }
+    return widen(((const uint16_t *)base)[i], f);
+}
+
+/* Store a binary32 value into element i of a storage-typed tensor, rounding once (nearest-even). */
+static void store_rounded(void *base, int64_t i, float v, int dtype, storage_format f)
+{
+    if (dtype == ORACLE_FP32) {
+        memcpy((unsigned char *)base + 4 * i, &v, 4);
+    } else {
+        ((uint16_t *)base)[i] = round_to_storage((double)v, f);
+    }
+}
+
 /*
  * fused_add_rmsnorm  (Table 1, Kernel 2):
  *     y = (x + r) / sqrt( (1/H) * ||x + r||^2 + eps )  (.)  w
@@ -135,28 +159,39 @@ uint16_t oracle_round_to_storage(double v, int dtype)
  *    square root, added to the mean of squares, as printed.
  *  - No rounding between the normalisation and the multiplication by w.
  */
-void oracle_fused_add_rmsnorm(const uint16_t *x, const uint16_t *r, const uint16_t *w,
+/* The one binary32 addition of the operation.  Operands of the 16-bit storage types have at most
+   11 significant bits, so their double sum rounded once to float is that addition; binary32
+   operands are added as floats. */
+static float add_binary32(double a, double b, int dtype)
+{
+    if (dtype == ORACLE_FP32) {
+        volatile float fa = (float)a, fb = (float)b;
+        volatile float s = fa + fb;
+        return s;
+    }
+    return (float)(a + b);
+}
+
+void oracle_fused_add_rmsnorm(const void *x, const void *r, const void *w,
                               int64_t T, int64_t H, float eps, int dtype,
-                              double *y_out, uint16_t *residual_out, int nthreads)
+                              double *y_out, void *residual_out, int nthreads)
 {
     storage_format f = format_of(dtype);
     if (nthreads < 1) nthreads = 1;
 #pragma omp parallel for num_threads(nthreads) schedule(static)
     for (int64_t t = 0; t < T; ++t) {
-        const uint16_t *xt = x + t * H;
-        const uint16_t *rt = r + t * H;
         double sum_sq = 0.0;
         for (int64_t j = 0; j < H; ++j) {
-            double s_exact = widen(xt[j], f) + widen(rt[j], f); /* exact in double */
-            double s = (double)(float)s_exact;                  /* binary32 add    */
+            double xv = load_value(x, t * H + j, dtype, f), rv = load_value(r, t * H + j, dtype, f);
+            double s = (double)add_binary32(xv, rv, dtype);
             sum_sq += s * s;
         }
         double denom = sqrt(sum_sq / (double)H + (double)eps);
         for (int64_t j = 0; j < H; ++j) {
-            double s_exact = widen(xt[j], f) + widen(rt[j], f);
-            float s32 = (float)s_exact;
-            residual_out[t * H + j] = round_to_storage((double)s32, f);
-            y_out[t * H + j] = (double)s32 / denom * widen(w[j], f);
+            double xv = load_value(x, t * H + j, dtype, f), rv = load_value(r, t * H + j, dtype, f);
+            float s32 = add_binary32(xv, rv, dtype);
+            store_rounded(residual_out, t * H + j, s32, dtype, f);
+            y_out[t * H + j] = (double)s32 / denom * load_value(w, j, dtype, f);
         }
     }
 }
@@ -180,17 +215,17 @@ static double silu(double z)
     return z / (1.0 + exp(-z));
 }
 
-void oracle_silu_and_mul(const uint16_t *input, int64_t T, int64_t D, int dtype,
+void oracle_silu_and_mul(const void *input, int64_t T, int64_t D, int dtype,
                          double *out, int nthreads)
 {
     storage_format f = format_of(dtype);
     if (nthreads < 1) nthreads = 1;
 #pragma omp parallel for num_threads(nthreads) schedule(static)
     for (int64_t t = 0; t < T; ++t) {
-        const uint16_t *row = input + t * 2 * D;
+        const int64_t row = t * 2 * D;
         for (int64_t i = 0; i < D; ++i) {
-            double a = widen(row[i], f);
-            double b = widen(row[D + i], f);
+            double a = load_value(input, row + i, dtype, f);
+            double b = load_value(input, row + D + i, dtype, f);
             out[t * D + i] = silu(a) * b;
         }
     }
@@ -214,8 +249,8 @@ void oracle_silu_and_mul(const uint16_t *input, int64_t T, int64_t D, int dtype,
  *    V_out = 0 and S_out = -inf.
  *  - +inf or NaN scores are outside the operation's domain: NaN out.
  */
-void oracle_merge_attn_states_lse(const uint16_t *v_a, const float *lse_a,
-                                  const uint16_t *v_b, const float *lse_b,
+void oracle_merge_attn_states_lse(const void *v_a, const float *lse_a,
+                                  const void *v_b, const float *lse_b,
                                   int64_t T, int64_t Hh, int64_t D, int dtype,
                                   double *v_out, double *lse_out, int nthreads)
 {
@@ -225,8 +260,7 @@ void oracle_merge_attn_states_lse(const uint16_t *v_a, const float *lse_a,
     for (int64_t th = 0; th < T * Hh; ++th) {
         double sa = (double)lse_a[th];
         double sb = (double)lse_b[th];
-        const uint16_t *va = v_a + th * D;
-        const uint16_t *vb = v_b + th * D;
+        const int64_t base = th * D;
         double *vo = v_out + th * D;
 
         if (isnan(sa) || isnan(sb) || sa == INFINITY || sb == INFINITY) {
@@ -245,8 +279,8 @@ void oracle_merge_attn_states_lse(const uint16_t *v_a, const float *lse_a,
         double denom = wa + wb;
         for (int64_t d = 0; d < D; ++d) {
             double num = 0.0;
-            if (wa != 0.0) num += wa * widen(va[d], f);
-            if (wb != 0.0) num += wb * widen(vb[d], f);
+            if (wa != 0.0) num += wa * load_value(v_a, base + d, dtype, f);
+            if (wb != 0.0) num += wb * load_value(v_b, base + d, dtype, f);
             vo[d] = num / denom;
         }
         lse_out[th] = m + log(denom);

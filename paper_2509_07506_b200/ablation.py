@@ -54,6 +54,13 @@ def load_library() -> ctypes.CDLL:
     return lib
 
 
+def _code16(t: torch.Tensor, name: str) -> int:
+    """dtype code of a 16-bit tensor (the design pairs are built for the 16-bit storage types only)."""
+    if t.dtype not in (torch.bfloat16, torch.float16):
+        raise TypeError(f"{name} must be bfloat16 or float16, got {t.dtype}")
+    return binding._code(t, name)
+
+
 def _raise(st: int, where: str) -> None:
     if st != binding.ASTRA_OK:
         raise binding.AstraError(st, where)
@@ -70,7 +77,7 @@ def astra_ablation_fused_add_rmsnorm(design: int, x, residual, weight, eps: floa
     T, H = x.shape
     _raise(load_library().astra_ablation_fused_add_rmsnorm(
         int(design), x.data_ptr(), residual.data_ptr(), weight.data_ptr(), T, H, float(eps),
-        binding._code(x, "x"), _stream(x, stream)), "astra_ablation_fused_add_rmsnorm")
+        _code16(x, "x"), _stream(x, stream)), "astra_ablation_fused_add_rmsnorm")
 
 
 def astra_ablation_silu_and_mul(design: int, out, input, stream=None) -> None:
@@ -79,7 +86,7 @@ def astra_ablation_silu_and_mul(design: int, out, input, stream=None) -> None:
             raise TypeError("contiguous CUDA tensors of one dtype expected")
     T, D = input.shape[0], input.shape[1] // 2
     _raise(load_library().astra_ablation_silu_and_mul(
-        int(design), out.data_ptr(), input.data_ptr(), T, D, binding._code(input, "input"),
+        int(design), out.data_ptr(), input.data_ptr(), T, D, _code16(input, "input"),
         _stream(input, stream)), "astra_ablation_silu_and_mul")
 
 
@@ -90,7 +97,7 @@ def astra_ablation_merge_attn_states_lse(design: int, v_out, lse_out, v_a, lse_a
     T, Hh, D = v_a.shape
     _raise(load_library().astra_ablation_merge_attn_states_lse(
         int(design), v_out.data_ptr(), lse_out.data_ptr(), v_a.data_ptr(), lse_a.data_ptr(), v_b.data_ptr(),
-        lse_b.data_ptr(), T, Hh, D, binding._code(v_a, "v_a"), _stream(v_a, stream)),
+        lse_b.data_ptr(), T, Hh, D, _code16(v_a, "v_a"), _stream(v_a, stream)),
         "astra_ablation_merge_attn_states_lse")
 
 

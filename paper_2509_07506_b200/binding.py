@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libastra.so
 
 ASTRA_BF16 = 0
 ASTRA_FP16 = 1
+ASTRA_FP32 = 2
 
 ASTRA_OK = 0
 ASTRA_ERR_NULL_POINTER = 1
@@ -37,7 +38,7 @@ EXPORTED_SYMBOLS = (
     "astra_status_string",
 )
 
-_DTYPE_CODE = {torch.bfloat16: ASTRA_BF16, torch.float16: ASTRA_FP16}
+_DTYPE_CODE = {torch.bfloat16: ASTRA_BF16, torch.float16: ASTRA_FP16, torch.float32: ASTRA_FP32}
 
 
 class AstraError(RuntimeError):
@@ -96,7 +97,7 @@ def _check(t: torch.Tensor, name: str, dtype=None, shape=None) -> None:
 
 def _code(t: torch.Tensor, name: str) -> int:
     if t.dtype not in _DTYPE_CODE:
-        raise TypeError(f"{name} must be bfloat16 or float16, got {t.dtype}")
+        raise TypeError(f"{name} must be bfloat16, float16 or float32, got {t.dtype}")
     return _DTYPE_CODE[t.dtype]
 
 

@@ -27,7 +27,7 @@ inline int64_t span_bytes(int64_t rows, int64_t width, int64_t pitch, int64_t el
     return ((rows - 1) * pitch + width) * elem;
 }
 
-// Do two [rows, width] tensors of 16-bit elements with the given row pitches share any element?
+// Do two [rows, width] tensors of 16-bit units with the given row pitches share any unit?
 // Exact when the pitches are equal (slices of one wider buffer: rows interleave without touching);
 // otherwise conservative (overlapping address spans count as overlap).
 inline bool pitched_overlap(const void *a, int64_t pitch_a, const void *b, int64_t pitch_b,
@@ -43,8 +43,8 @@ inline bool pitched_overlap(const void *a, int64_t pitch_a, const void *b, int64
     return hits_k || hits_k1;
 }
 
-// Largest vector width (in 16-bit elements, a power of two up to max_vec) that divides every extent
-// in `extents` and to which every pointer is aligned.  Row starts are multiples of the pitches, so
+// Largest vector width (in 16-bit units, a power of two up to max_vec) that divides every extent
+// (given in units) and to which every pointer is aligned.  Row starts are multiples of the pitches, so
 // every vector access of every row is then naturally aligned.
 struct VecPick {
     int vec;
@@ -95,15 +95,31 @@ inline void launch(void (*kernel)(KArgs...), unsigned grid, unsigned block, cuda
 constexpr int64_t kMaxVecsPerLaunch = ASTRA_MAX_VECS_PER_LAUNCH;
 constexpr int64_t kInt64Max = 9223372036854775807ll;
 
-inline bool valid_dtype(astra_dtype_t d) { return d == ASTRA_BF16 || d == ASTRA_FP16; }
+inline bool valid_dtype(astra_dtype_t d) { return d == ASTRA_BF16 || d == ASTRA_FP16 || d == ASTRA_FP32; }
+
+// All value tensors are addressed in 16-bit units inside the library: an element is 1 unit for the
+// 16-bit storage types and 2 for binary32.  Entry points validate in elements, then scale widths and
+// pitches to units once; kernels turn a vector of UV units back into UV / UNITS elements.
+inline int64_t units_per_elem(astra_dtype_t d) { return d == ASTRA_FP32 ? 2 : 1; }
+
+// Runs CALL with the compile-time constant DT set to the runtime dtype (already validated).
+#define ASTRA_FOR_DTYPE(dtype, CALL)                                        \
+    do {                                                                    \
+        if ((dtype) == ASTRA_BF16) { constexpr int DT = ASTRA_BF16; CALL; } \
+        else if ((dtype) == ASTRA_FP16) { constexpr int DT = ASTRA_FP16; CALL; } \
+        else { constexpr int DT = ASTRA_FP32; CALL; }                       \
+    } while (0)
 
 // ---------------------------------------------------------------------------------------------
 // silu_and_mul
 // ---------------------------------------------------------------------------------------------
-template <int DT, int VEC, int UNROLL, int THREADS>
+// D, the pitches and the pointers are in 16-bit units; UVEC is the vector width in units.
+template <int DT, int UVEC, int UNROLL, int THREADS>
 void launch_silu(uint16_t *out, const uint16_t *gate, const uint16_t *up, int64_t T, int64_t D,
                  int64_t out_pitch, int64_t gate_pitch, int64_t up_pitch, cudaStream_t stream) {
-    const int64_t nvec = D / VEC;
+  if constexpr (UVEC >= Storage<DT>::UNITS) {
+    constexpr int VEC = UVEC / Storage<DT>::UNITS;
+    const int64_t nvec = D / UVEC;
     const int64_t rows_per_launch = kMaxVecsPerLaunch / nvec;
     for (int64_t t0 = 0; t0 < T; t0 += rows_per_launch) {
         const int64_t rows = (T - t0 < rows_per_launch) ? (T - t0) : rows_per_launch;
@@ -114,6 +130,7 @@ void launch_silu(uint16_t *out, const uint16_t *gate, const uint16_t *up, int64_
                out + t0 * out_pitch, gate + t0 * gate_pitch, up + t0 * up_pitch, total,
                FastDiv::make(static_cast<uint32_t>(nvec)), out_pitch, gate_pitch, up_pitch);
     }
+  }
 }
 
 template <int DT>
@@ -141,29 +158,31 @@ astra_status_t silu_entry(void *out, const void *gate, const void *up, int64_t T
     const int64_t max_pitch = out_pitch > gate_pitch ? (out_pitch > up_pitch ? out_pitch : up_pitch)
                                                      : (gate_pitch > up_pitch ? gate_pitch : up_pitch);
     if (T > 0 && max_pitch > kInt64Max / 4 / T) return ASTRA_ERR_BAD_SHAPE;
-    if (!aligned(out, 2) || !aligned(gate, 2) || !aligned(up, 2)) return ASTRA_ERR_MISALIGNED;
+    const int64_t U = units_per_elem(dtype);
+    const size_t eb = static_cast<size_t>(2 * U);
+    if (!aligned(out, eb) || !aligned(gate, eb) || !aligned(up, eb)) return ASTRA_ERR_MISALIGNED;
     if (T == 0) return ASTRA_OK;
-    if (pitched_overlap(out, out_pitch, gate, gate_pitch, T, D) ||
-        pitched_overlap(out, out_pitch, up, up_pitch, T, D))
+    const int64_t Du = D * U, opu = out_pitch * U, gpu = gate_pitch * U, upu = up_pitch * U;  // in units
+    if (pitched_overlap(out, opu, gate, gpu, T, Du) || pitched_overlap(out, opu, up, upu, T, Du))
         return ASTRA_ERR_OVERLAP;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     uint16_t *op = static_cast<uint16_t *>(out);
     const uint16_t *gp = static_cast<const uint16_t *>(gate), *upp = static_cast<const uint16_t *>(up);
-    if (dtype == ASTRA_BF16)
-        dispatch_silu<ASTRA_BF16>(op, gp, upp, T, D, out_pitch, gate_pitch, up_pitch, stream);
-    else
-        dispatch_silu<ASTRA_FP16>(op, gp, upp, T, D, out_pitch, gate_pitch, up_pitch, stream);
+    ASTRA_FOR_DTYPE(dtype, dispatch_silu<DT>(op, gp, upp, T, Du, opu, gpu, upu, stream));
     return launch_status();
 }
 
 // ---------------------------------------------------------------------------------------------
 // merge_attn_states_lse
 // ---------------------------------------------------------------------------------------------
-template <int DT, int VEC, int UNROLL, int THREADS>
+// D and the value pointers are in 16-bit units; UVEC is the vector width in units.
+template <int DT, int UVEC, int UNROLL, int THREADS>
 void launch_merge(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
                   const uint16_t *v_b, const float *lse_b, int64_t rows_total, int64_t D,
                   cudaStream_t stream) {
-    const int64_t nvec = D / VEC;
+  if constexpr (UVEC >= Storage<DT>::UNITS) {
+    constexpr int VEC = UVEC / Storage<DT>::UNITS;
+    const int64_t nvec = D / UVEC;
     const int64_t rows_per_launch = kMaxVecsPerLaunch / nvec;
     for (int64_t r0 = 0; r0 < rows_total; r0 += rows_per_launch) {
         const int64_t rows = (rows_total - r0 < rows_per_launch) ? (rows_total - r0) : rows_per_launch;
@@ -174,6 +193,7 @@ void launch_merge(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const fl
                v_out + r0 * D, lse_out ? lse_out + r0 : nullptr, v_a + r0 * D, lse_a + r0, v_b + r0 * D,
                lse_b + r0, total, FastDiv::make(static_cast<uint32_t>(nvec)));
     }
+  }
 }
 
 template <int DT>
@@ -190,11 +210,13 @@ void dispatch_merge(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const 
     }
 }
 
-template <int DT, int VEC, int UNROLL, int THREADS>
+template <int DT, int UVEC, int UNROLL, int THREADS>
 void launch_merge_strided(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
                           const uint16_t *v_b, const float *lse_b, int64_t rows_total, int64_t Hh,
                           int64_t D, const MergeStrides &st, cudaStream_t stream) {
-    const int64_t nvec = D / VEC;
+  if constexpr (UVEC >= Storage<DT>::UNITS) {
+    constexpr int VEC = UVEC / Storage<DT>::UNITS;
+    const int64_t nvec = D / UVEC;
     const int64_t rows_per_launch = kMaxVecsPerLaunch / nvec;
     for (int64_t r0 = 0; r0 < rows_total; r0 += rows_per_launch) {
         const int64_t rows = (rows_total - r0 < rows_per_launch) ? (rows_total - r0) : rows_per_launch;
@@ -205,6 +227,7 @@ void launch_merge_strided(uint16_t *v_out, float *lse_out, const uint16_t *v_a, 
                v_out, lse_out, v_a, lse_a, v_b, lse_b, total, static_cast<uint32_t>(r0),
                FastDiv::make(static_cast<uint32_t>(nvec)), FastDiv::make(static_cast<uint32_t>(Hh)), st);
     }
+  }
 }
 
 template <int DT>
@@ -246,36 +269,42 @@ inline bool rows_disjoint(int64_t T, int64_t Hh, int64_t W, int64_t st, int64_t 
 // ---------------------------------------------------------------------------------------------
 constexpr int kMaxGridX = ASTRA_MAX_ROWS_PER_LAUNCH;
 
-// Most elements of a row one thread keeps in registers: 64 with vector accesses, 16 on the scalar
-// path (each element then also costs three separate packed-input registers).
-constexpr int rmsnorm_max_elems_per_thread(int vec) { return vec == 1 ? 16 : 64; }
+// Most 16-bit units of a row one thread keeps in registers: 64 with vector accesses, 16 on the
+// scalar path (each element then also costs three separate packed-input registers).
+constexpr int rmsnorm_max_units_per_thread(int uvec) { return uvec == 1 ? 16 : 64; }
 
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
-template <int DT, int VEC, int VPT>
+template <int DT, int UVEC, int VPT>
 inline void launch_rmsnorm_reg(unsigned rows, int threads, cudaStream_t stream, const RmsnormOperands &op,
                                const uint16_t *w, int H, float eps, float inv_H) {
     // wider combinations than the per-thread cap are never selected and are not instantiated
-    if constexpr (VEC * VPT <= rmsnorm_max_elems_per_thread(VEC))
-        launch(fused_add_rmsnorm_reg_kernel<DT, VEC, VPT>, rows, threads, stream, op, w, H, eps, inv_H);
+    if constexpr (UVEC * VPT <= rmsnorm_max_units_per_thread(UVEC))
+        launch(fused_add_rmsnorm_reg_kernel<DT, UVEC / Storage<DT>::UNITS, VPT>, rows, threads, stream, op, w, H,
+               eps, inv_H);
 }
 
 // Register-resident rows: VPT vectors per thread with blockDim = ceil(nvec / VPT) rounded up to a warp.
-// 16 elements per thread (32 bytes of x and of r in flight per thread) with 256..1024 threads
-// measured best; up to 64 elements per thread are used for wider rows, with the block size capped
-// so the row still fits the register file.  Rows wider than that take the two-sweep kernel.
-template <int DT, int VEC>
+// 16 units per thread (32 bytes of x and of r in flight per thread) with 256..1024 threads measured
+// best; up to 64 units per thread are used for wider rows, with the block size capped so the row
+// still fits the register file.  Rows wider than that take the two-sweep kernel.
+// H is in elements; the operands' pointers and pitches are in 16-bit units; UVEC is the vector width
+// in units.
+template <int DT, int UVEC>
 void launch_rmsnorm(RmsnormOperands op, const uint16_t *w, int64_t T, int H, float eps, cudaStream_t stream) {
+  if constexpr (UVEC >= Storage<DT>::UNITS) {
+    constexpr int VEC = UVEC / Storage<DT>::UNITS;
+    constexpr int kMaxVpt = rmsnorm_max_units_per_thread(UVEC) / UVEC;
     const int nvec = H / VEC;
     const float inv_H = 1.0f / static_cast<float>(H);
-    // start at 16 elements per thread; widen the per-thread share only if the row needs more
-    // threads than that share allows, narrow it if the block would fall under 128 threads
-    int vpt = 16 / VEC < 1 ? 1 : 16 / VEC;
+    // start at 16 units per thread; widen the per-thread share only if the row needs more threads
+    // than that share allows, narrow it if the block would fall under 128 threads
+    int vpt = 16 / UVEC < 1 ? 1 : 16 / UVEC;
     auto threads_for = [&](int v) { return round_up((nvec + v - 1) / v, 32); };
-    while (vpt < rmsnorm_max_elems_per_thread(VEC) / VEC && threads_for(vpt) > rmsnorm_reg_max_threads(VEC, vpt)) vpt <<= 1;
+    while (vpt < kMaxVpt && threads_for(vpt) > rmsnorm_reg_max_threads(UVEC * vpt)) vpt <<= 1;
     while (vpt > 1 && threads_for(vpt) < 128) vpt >>= 1;
     const int threads = threads_for(vpt);
-    const bool fits = threads <= rmsnorm_reg_max_threads(VEC, vpt);
+    const bool fits = threads <= rmsnorm_reg_max_threads(UVEC * vpt);
     for (int64_t t0 = 0; t0 < T; t0 += kMaxGridX) {
         const unsigned rows = static_cast<unsigned>(T - t0 < kMaxGridX ? T - t0 : kMaxGridX);
         RmsnormOperands o = op;
@@ -288,23 +317,24 @@ void launch_rmsnorm(RmsnormOperands op, const uint16_t *w, int64_t T, int H, flo
             continue;
         }
         switch (vpt) {
-            case 1: launch_rmsnorm_reg<DT, VEC, 1>(rows, threads, stream, o, w, H, eps, inv_H); break;
-            case 2: launch_rmsnorm_reg<DT, VEC, 2>(rows, threads, stream, o, w, H, eps, inv_H); break;
-            case 4: launch_rmsnorm_reg<DT, VEC, 4>(rows, threads, stream, o, w, H, eps, inv_H); break;
-            case 8: launch_rmsnorm_reg<DT, VEC, 8>(rows, threads, stream, o, w, H, eps, inv_H); break;
-            case 16: launch_rmsnorm_reg<DT, VEC, 16>(rows, threads, stream, o, w, H, eps, inv_H); break;
-            case 32: launch_rmsnorm_reg<DT, VEC, 32>(rows, threads, stream, o, w, H, eps, inv_H); break;
-            default: launch_rmsnorm_reg<DT, VEC, 64>(rows, threads, stream, o, w, H, eps, inv_H); break;
+            case 1: launch_rmsnorm_reg<DT, UVEC, 1>(rows, threads, stream, o, w, H, eps, inv_H); break;
+            case 2: launch_rmsnorm_reg<DT, UVEC, 2>(rows, threads, stream, o, w, H, eps, inv_H); break;
+            case 4: launch_rmsnorm_reg<DT, UVEC, 4>(rows, threads, stream, o, w, H, eps, inv_H); break;
+            case 8: launch_rmsnorm_reg<DT, UVEC, 8>(rows, threads, stream, o, w, H, eps, inv_H); break;
+            case 16: launch_rmsnorm_reg<DT, UVEC, 16>(rows, threads, stream, o, w, H, eps, inv_H); break;
+            case 32: launch_rmsnorm_reg<DT, UVEC, 32>(rows, threads, stream, o, w, H, eps, inv_H); break;
+            default: launch_rmsnorm_reg<DT, UVEC, 64>(rows, threads, stream, o, w, H, eps, inv_H); break;
         }
     }
+  }
 }
 
 template <int DT>
 void dispatch_rmsnorm(const RmsnormOperands &op, const uint16_t *w, int64_t T, int H, float eps,
                       cudaStream_t stream) {
-    const int vec = VecPick(8).extent(H).extent(op.x_pitch).extent(op.r_pitch).extent(op.y_pitch)
-                        .extent(op.r_out_pitch).pointer(op.x).pointer(op.r).pointer(op.y).pointer(op.r_out)
-                        .pointer(w).vec;
+    const int vec = VecPick(8).extent(static_cast<int64_t>(H) * Storage<DT>::UNITS).extent(op.x_pitch)
+                        .extent(op.r_pitch).extent(op.y_pitch).extent(op.r_out_pitch).pointer(op.x)
+                        .pointer(op.r).pointer(op.y).pointer(op.r_out).pointer(w).vec;
     switch (vec) {
         case 8: launch_rmsnorm<DT, 8>(op, w, T, H, eps, stream); break;
         case 4: launch_rmsnorm<DT, 4>(op, w, T, H, eps, stream); break;
@@ -326,20 +356,28 @@ astra_status_t rmsnorm_entry(void *y, void *residual_out, const void *x, const v
     if (x_pitch > max_pitch) max_pitch = x_pitch;
     if (r_pitch > max_pitch) max_pitch = r_pitch;
     if (T > 0 && max_pitch > kInt64Max / 4 / T) return ASTRA_ERR_BAD_SHAPE;
-    if (!aligned(y, 2) || !aligned(residual_out, 2) || !aligned(x, 2) || !aligned(residual, 2) ||
-        !aligned(weight, 2))
+    const int64_t U = units_per_elem(dtype);
+    const size_t eb = static_cast<size_t>(2 * U);
+    if (!aligned(y, eb) || !aligned(residual_out, eb) || !aligned(x, eb) || !aligned(residual, eb) ||
+        !aligned(weight, eb))
         return ASTRA_ERR_MISALIGNED;
     if (T == 0) return ASTRA_OK;
+    // from here on widths and pitches are in 16-bit units
+    const int64_t Hu = H * U;
+    y_pitch *= U;
+    ro_pitch *= U;
+    x_pitch *= U;
+    r_pitch *= U;
     const bool y_is_x = (y == x && y_pitch == x_pitch);
     const bool ro_is_r = (residual_out == residual && ro_pitch == r_pitch);
     // the weight is one row: compare it against every output as a [T, H] tensor of pitch 0 would be
     // wrong (pitch < width), so use the outputs' spans for it
-    const int64_t sy = span_bytes(T, H, y_pitch, 2), sro = span_bytes(T, H, ro_pitch, 2), sw = H * 2;
-    if ((!y_is_x && pitched_overlap(y, y_pitch, x, x_pitch, T, H)) ||
-        pitched_overlap(y, y_pitch, residual, r_pitch, T, H) ||
-        pitched_overlap(y, y_pitch, residual_out, ro_pitch, T, H) || overlaps(y, sy, weight, sw) ||
-        (!ro_is_r && pitched_overlap(residual_out, ro_pitch, residual, r_pitch, T, H)) ||
-        pitched_overlap(residual_out, ro_pitch, x, x_pitch, T, H) || overlaps(residual_out, sro, weight, sw))
+    const int64_t sy = span_bytes(T, Hu, y_pitch, 2), sro = span_bytes(T, Hu, ro_pitch, 2), sw = Hu * 2;
+    if ((!y_is_x && pitched_overlap(y, y_pitch, x, x_pitch, T, Hu)) ||
+        pitched_overlap(y, y_pitch, residual, r_pitch, T, Hu) ||
+        pitched_overlap(y, y_pitch, residual_out, ro_pitch, T, Hu) || overlaps(y, sy, weight, sw) ||
+        (!ro_is_r && pitched_overlap(residual_out, ro_pitch, residual, r_pitch, T, Hu)) ||
+        pitched_overlap(residual_out, ro_pitch, x, x_pitch, T, Hu) || overlaps(residual_out, sro, weight, sw))
         return ASTRA_ERR_OVERLAP;
     RmsnormOperands op;
     op.x = static_cast<const uint16_t *>(x);
@@ -352,10 +390,7 @@ astra_status_t rmsnorm_entry(void *y, void *residual_out, const void *x, const v
     op.r_out_pitch = ro_pitch;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const uint16_t *wp = static_cast<const uint16_t *>(weight);
-    if (dtype == ASTRA_BF16)
-        dispatch_rmsnorm<ASTRA_BF16>(op, wp, T, static_cast<int>(H), eps, stream);
-    else
-        dispatch_rmsnorm<ASTRA_FP16>(op, wp, T, static_cast<int>(H), eps, stream);
+    ASTRA_FOR_DTYPE(dtype, dispatch_rmsnorm<DT>(op, wp, T, static_cast<int>(H), eps, stream));
     return launch_status();
 }
 
@@ -381,7 +416,7 @@ astra_status_t astra_silu_and_mul(void *out, const void *input, int64_t T, int64
                                   astra_dtype_t dtype, void *cuda_stream) {
     if (!input) return ASTRA_ERR_NULL_POINTER;
     if (D <= 0 || D > 1073741823ll) return ASTRA_ERR_BAD_SHAPE;
-    const void *up = static_cast<const uint16_t *>(input) + D;
+    const void *up = static_cast<const uint16_t *>(input) + D * units_per_elem(dtype);
     return silu_entry(out, input, up, T, D, D, 2 * D, 2 * D, dtype, cuda_stream);
 }
 
@@ -399,12 +434,15 @@ astra_status_t astra_merge_attn_states_lse(void *v_out, float *lse_out, const vo
     if (!valid_dtype(dtype)) return ASTRA_ERR_BAD_DTYPE;
     if (T < 0 || Hh <= 0 || D <= 0 || D > 2147483647ll) return ASTRA_ERR_BAD_SHAPE;
     if (T > 0 && (Hh > kInt64Max / 4 / T || D > kInt64Max / 4 / (T * Hh))) return ASTRA_ERR_BAD_SHAPE;
-    if (!aligned(v_out, 2) || !aligned(v_a, 2) || !aligned(v_b, 2) || !aligned(lse_a, 4) ||
+    const int64_t U = units_per_elem(dtype);
+    const size_t eb = static_cast<size_t>(2 * U);
+    if (!aligned(v_out, eb) || !aligned(v_a, eb) || !aligned(v_b, eb) || !aligned(lse_a, 4) ||
         !aligned(lse_b, 4) || (lse_out && !aligned(lse_out, 4)))
         return ASTRA_ERR_MISALIGNED;
     if (T == 0) return ASTRA_OK;
     const int64_t rows = T * Hh;
-    const int64_t vbytes = rows * D * 2, sbytes = rows * 4;
+    const int64_t Du = D * U;  // row width in 16-bit units
+    const int64_t vbytes = rows * Du * 2, sbytes = rows * 4;
     if ((v_out != v_a && overlaps(v_out, vbytes, v_a, vbytes)) ||
         (v_out != v_b && overlaps(v_out, vbytes, v_b, vbytes)))
         return ASTRA_ERR_OVERLAP;
@@ -417,10 +455,7 @@ astra_status_t astra_merge_attn_states_lse(void *v_out, float *lse_out, const vo
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     uint16_t *vo = static_cast<uint16_t *>(v_out);
     const uint16_t *va = static_cast<const uint16_t *>(v_a), *vb = static_cast<const uint16_t *>(v_b);
-    if (dtype == ASTRA_BF16)
-        dispatch_merge<ASTRA_BF16>(vo, lse_out, va, lse_a, vb, lse_b, rows, D, stream);
-    else
-        dispatch_merge<ASTRA_FP16>(vo, lse_out, va, lse_a, vb, lse_b, rows, D, stream);
+    ASTRA_FOR_DTYPE(dtype, dispatch_merge<DT>(vo, lse_out, va, lse_a, vb, lse_b, rows, Du, stream));
     return launch_status();
 }
 
@@ -438,22 +473,25 @@ astra_status_t astra_merge_attn_states_lse_ex(void *v_out, float *lse_out, const
         const int64_t steps = (i % 2 == 0 ? T : Hh) - 1;
         if (strides[i] < 0 || (steps > 0 && strides[i] > (1ll << 60) / steps)) return ASTRA_ERR_BAD_SHAPE;
     }
+    const int64_t U = units_per_elem(dtype);
+    const size_t eb = static_cast<size_t>(2 * U);
+    const int64_t Du = D * U;  // row width and value strides in 16-bit units from here on
     MergeStrides st;
-    st.va_t = strides[0]; st.va_h = strides[1]; st.vb_t = strides[2]; st.vb_h = strides[3];
-    st.vo_t = strides[4]; st.vo_h = strides[5]; st.sa_t = strides[6]; st.sa_h = strides[7];
+    st.va_t = strides[0] * U; st.va_h = strides[1] * U; st.vb_t = strides[2] * U; st.vb_h = strides[3] * U;
+    st.vo_t = strides[4] * U; st.vo_h = strides[5] * U; st.sa_t = strides[6]; st.sa_h = strides[7];
     st.sb_t = strides[8]; st.sb_h = strides[9];
     st.so_t = lse_out ? strides[10] : 0;
     st.so_h = lse_out ? strides[11] : 0;
-    if (!aligned(v_out, 2) || !aligned(v_a, 2) || !aligned(v_b, 2) || !aligned(lse_a, 4) ||
+    if (!aligned(v_out, eb) || !aligned(v_a, eb) || !aligned(v_b, eb) || !aligned(lse_a, 4) ||
         !aligned(lse_b, 4) || (lse_out && !aligned(lse_out, 4)))
         return ASTRA_ERR_MISALIGNED;
     if (T == 0) return ASTRA_OK;
     // written tensors must have non-overlapping rows; read tensors may broadcast (stride 0)
-    if (!rows_disjoint(T, Hh, D, st.vo_t, st.vo_h)) return ASTRA_ERR_BAD_SHAPE;
+    if (!rows_disjoint(T, Hh, Du, st.vo_t, st.vo_h)) return ASTRA_ERR_BAD_SHAPE;
     if (lse_out && !rows_disjoint(T, Hh, 1, st.so_t, st.so_h)) return ASTRA_ERR_BAD_SHAPE;
-    const int64_t bva = strided_extent(T, Hh, D, st.va_t, st.va_h) * 2;
-    const int64_t bvb = strided_extent(T, Hh, D, st.vb_t, st.vb_h) * 2;
-    const int64_t bvo = strided_extent(T, Hh, D, st.vo_t, st.vo_h) * 2;
+    const int64_t bva = strided_extent(T, Hh, Du, st.va_t, st.va_h) * 2;
+    const int64_t bvb = strided_extent(T, Hh, Du, st.vb_t, st.vb_h) * 2;
+    const int64_t bvo = strided_extent(T, Hh, Du, st.vo_t, st.vo_h) * 2;
     const int64_t bsa = strided_extent(T, Hh, 1, st.sa_t, st.sa_h) * 4;
     const int64_t bsb = strided_extent(T, Hh, 1, st.sb_t, st.sb_h) * 4;
     const int64_t bso = lse_out ? strided_extent(T, Hh, 1, st.so_t, st.so_h) * 4 : 0;
@@ -470,10 +508,7 @@ astra_status_t astra_merge_attn_states_lse_ex(void *v_out, float *lse_out, const
     uint16_t *vo = static_cast<uint16_t *>(v_out);
     const uint16_t *va = static_cast<const uint16_t *>(v_a), *vb = static_cast<const uint16_t *>(v_b);
     const int64_t rows = T * Hh;
-    if (dtype == ASTRA_BF16)
-        dispatch_merge_strided<ASTRA_BF16>(vo, lse_out, va, lse_a, vb, lse_b, rows, Hh, D, st, stream);
-    else
-        dispatch_merge_strided<ASTRA_FP16>(vo, lse_out, va, lse_a, vb, lse_b, rows, Hh, D, st, stream);
+    ASTRA_FOR_DTYPE(dtype, dispatch_merge_strided<DT>(vo, lse_out, va, lse_a, vb, lse_b, rows, Hh, Du, st, stream));
     return launch_status();
 }
 

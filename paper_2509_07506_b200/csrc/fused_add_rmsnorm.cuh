@@ -16,7 +16,7 @@ namespace astra {
 
 constexpr int kMaxWarps = 32;
 
-// Row-addressed operands.  Pitches are in elements.  y may be exactly x and r_out exactly r (the
+// Row-addressed operands.  Pointers and pitches are in 16-bit units.  y may be exactly x and r_out exactly r (the
 // in-place form); each thread reads the vectors it later overwrites, so that aliasing is safe.
 struct RmsnormOperands {
     const uint16_t *x;
@@ -42,23 +42,27 @@ __device__ __forceinline__ float block_sum(float v, float *slots) {
 }
 
 // Largest block the register-resident kernel may be launched with, by vectors per thread: the
-// row's binary32 sums (VPT * VEC registers) plus its packed inputs must fit the register file.
-__host__ __device__ constexpr int rmsnorm_reg_max_threads(int vec, int vpt) {
-    return vec * vpt <= 16 ? 1024 : (vec * vpt <= 32 ? 512 : 256);
+// row's binary32 sums plus its packed inputs (counted in 16-bit units per thread) must fit the
+// register file.
+__host__ __device__ constexpr int rmsnorm_reg_max_threads(int units_per_thread) {
+    return units_per_thread <= 16 ? 1024 : (units_per_thread <= 32 ? 512 : 256);
 }
 
 // Register-resident row: thread i owns vectors i, i + blockDim.x, ... (at most VPT of them).
-// Requires nvec = H / VEC <= VPT * blockDim.x and blockDim.x <= rmsnorm_reg_max_threads(VEC, VPT).
+// Requires nvec = H / VEC <= VPT * blockDim.x and blockDim.x <= rmsnorm_reg_max_threads(VEC * VPT * UNITS).
 // EARLY_W issues the weight loads before the reduction instead of after it (measured: no faster,
 // and it costs the registers that decide occupancy).  MINB is the minimum number of resident blocks
-// the register allocation must allow; with 16 elements per thread MINB = 2 caps the kernel at 32
-// registers, i.e. full occupancy for every block size, which is worth 5 % at [16384, 8192] and
-// 27 % at [512, 14336] (896-thread blocks: two per SM instead of one).
+// the register allocation must allow; with 16 units per thread in at most four vectors MINB = 2
+// caps the kernel at 32 registers, i.e. full occupancy for every block size, which is worth 5 % at
+// [16384, 8192] and 27 % at [512, 14336] (896-thread blocks: two per SM instead of one).  The
+// four-vector form (8-byte accesses, e.g. H = 4100) spills three registers under the cap and still
+// measured fastest; with eight or sixteen narrower vectors the spills grow, so no cap there.
 template <int DT, int VEC, int VPT, Ld LDH = Ld::Stream, St STH = St::Stream, bool EARLY_W = false,
-          int MINB = (VEC * VPT <= 16 ? 2 : 1)>
-__global__ void __launch_bounds__(rmsnorm_reg_max_threads(VEC, VPT), MINB)
+          int MINB = ((VEC * VPT * Storage<DT>::UNITS <= 16 && VPT <= 4) ? 2 : 1)>
+__global__ void __launch_bounds__(rmsnorm_reg_max_threads(VEC * VPT * Storage<DT>::UNITS), MINB)
 fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ weight,
                              int H, float eps, float inv_H) {
+    constexpr int UV = VEC * Storage<DT>::UNITS;  // 16-bit units per vector
     __shared__ float slots[kMaxWarps];
     const int nvec = H / VEC;
     const int64_t row = blockIdx.x;
@@ -69,21 +73,21 @@ fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ we
     grid_dependency_wait();
     grid_launch_dependents();
 
-    Pack<VEC> px[VPT], pr[VPT], pw[VPT];
+    Pack<UV> px[VPT], pr[VPT], pw[VPT];
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
         const int v = threadIdx.x + i * blockDim.x;
         if (v < nvec) {
             // x and residual may be rewritten by this same thread below: coherent loads, not .nc
-            px[i] = load<VEC, LDH>(xr + v * VEC);
-            pr[i] = load<VEC, LDH>(rr + v * VEC);
+            px[i] = load<UV, LDH>(xr + v * UV);
+            pr[i] = load<UV, LDH>(rr + v * UV);
         }
     }
     if constexpr (EARLY_W) {
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
             const int v = threadIdx.x + i * blockDim.x;
-            if (v < nvec) pw[i] = load<VEC, Ld::Keep>(weight + v * VEC);
+            if (v < nvec) pw[i] = load<UV, Ld::Keep>(weight + v * UV);
         }
     }
 
@@ -101,7 +105,7 @@ fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ we
                 s[i][k] = fx[k] + fr[k];  // the one binary32 add
                 acc = fmaf(s[i][k], s[i][k], acc);
             }
-            store<VEC, STH>(ror + v * VEC, narrow<DT, VEC>(s[i]));
+            store<UV, STH>(ror + v * UV, narrow<DT, VEC>(s[i]));
         }
     }
 
@@ -109,7 +113,7 @@ fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ we
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
             const int v = threadIdx.x + i * blockDim.x;
-            if (v < nvec) pw[i] = load<VEC, Ld::Keep>(weight + v * VEC);
+            if (v < nvec) pw[i] = load<UV, Ld::Keep>(weight + v * UV);
         }
     }
     const float total = block_sum(acc, slots);
@@ -123,7 +127,7 @@ fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ we
             widen<DT, VEC>(pw[i], fw);
 #pragma unroll
             for (int k = 0; k < VEC; ++k) fy[k] = s[i][k] * rstd * fw[k];
-            store<VEC, STH>(yr + v * VEC, narrow<DT, VEC>(fy));
+            store<UV, STH>(yr + v * UV, narrow<DT, VEC>(fy));
         }
     }
 }
@@ -136,6 +140,7 @@ template <int DT, int VEC>
 __global__ void fused_add_rmsnorm_twopass_kernel(RmsnormOperands op,
                                                  const uint16_t *__restrict__ weight,
                                                  int H, float eps, float inv_H) {
+    constexpr int UV = VEC * Storage<DT>::UNITS;  // 16-bit units per vector
     __shared__ float slots[kMaxWarps];
     const int nvec = H / VEC;
     const int64_t row = blockIdx.x;
@@ -149,8 +154,8 @@ __global__ void fused_add_rmsnorm_twopass_kernel(RmsnormOperands op,
     float acc = 0.f;
     for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
         float fx[VEC], fr[VEC];
-        widen<DT, VEC>(load<VEC, Ld::Stream>(xr + v * VEC), fx);
-        widen<DT, VEC>(load<VEC, Ld::Stream>(rr + v * VEC), fr);
+        widen<DT, VEC>(load<UV, Ld::Stream>(xr + v * UV), fx);
+        widen<DT, VEC>(load<UV, Ld::Stream>(rr + v * UV), fr);
 #pragma unroll
         for (int k = 0; k < VEC; ++k) {
             const float s = fx[k] + fr[k];
@@ -162,16 +167,16 @@ __global__ void fused_add_rmsnorm_twopass_kernel(RmsnormOperands op,
 
     for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
         float fx[VEC], fr[VEC], fw[VEC], fs[VEC], fy[VEC];
-        widen<DT, VEC>(load<VEC, Ld::Stream>(xr + v * VEC), fx);
-        widen<DT, VEC>(load<VEC, Ld::Stream>(rr + v * VEC), fr);
-        widen<DT, VEC>(load<VEC, Ld::Keep>(weight + v * VEC), fw);
+        widen<DT, VEC>(load<UV, Ld::Stream>(xr + v * UV), fx);
+        widen<DT, VEC>(load<UV, Ld::Stream>(rr + v * UV), fr);
+        widen<DT, VEC>(load<UV, Ld::Keep>(weight + v * UV), fw);
 #pragma unroll
         for (int k = 0; k < VEC; ++k) {
             fs[k] = fx[k] + fr[k];
             fy[k] = fs[k] * rstd * fw[k];
         }
-        store<VEC, St::Stream>(ror + v * VEC, narrow<DT, VEC>(fs));
-        store<VEC, St::Stream>(yr + v * VEC, narrow<DT, VEC>(fy));
+        store<UV, St::Stream>(ror + v * UV, narrow<DT, VEC>(fs));
+        store<UV, St::Stream>(yr + v * UV, narrow<DT, VEC>(fy));
     }
 }
 

@@ -48,7 +48,8 @@ __device__ __forceinline__ MergeWeights merge_weights(float sa, float sb) {
     return r;
 }
 
-// Strides (in elements) of one [T, Hh, D] value tensor or one [T, Hh] score tensor; D is contiguous.
+// Strides of one [T, Hh, D] value tensor (in 16-bit units) or one [T, Hh] score tensor (in floats);
+// D is contiguous.
 struct MergeStrides {
     int64_t va_t, va_h, vb_t, vb_h, vo_t, vo_h;  // values: token and head strides
     int64_t sa_t, sa_h, sb_t, sb_h, so_t, so_h;  // scores: token and head strides
@@ -61,10 +62,11 @@ merge_attn_states_lse_kernel(uint16_t *v_out, float *lse_out,
                              const uint16_t *v_a, const float *lse_a,
                              const uint16_t *v_b, const float *lse_b,
                              uint32_t total_vecs, FastDiv nvec) {
+    constexpr int UV = VEC * Storage<DT>::UNITS;  // 16-bit units per vector
     const uint32_t base = blockIdx.x * (THREADS * UNROLL) + threadIdx.x;
     grid_dependency_wait();
     grid_launch_dependents();
-    Pack<VEC> a[UNROLL], b[UNROLL];
+    Pack<UV> a[UNROLL], b[UNROLL];
     float sa[UNROLL], sb[UNROLL];
     uint32_t row[UNROLL];
 #pragma unroll
@@ -74,8 +76,8 @@ merge_attn_states_lse_kernel(uint16_t *v_out, float *lse_out,
             row[j] = nvec.div(v);
             // v_out may be exactly v_a or v_b, so these are ordinary (coherent) loads; the thread
             // that reads a vector is the only one that writes it
-            a[j] = load<VEC, LDH>(v_a + static_cast<int64_t>(v) * VEC);
-            b[j] = load<VEC, LDH>(v_b + static_cast<int64_t>(v) * VEC);
+            a[j] = load<UV, LDH>(v_a + static_cast<int64_t>(v) * UV);
+            b[j] = load<UV, LDH>(v_b + static_cast<int64_t>(v) * UV);
             sa[j] = lse_a[row[j]];
             sb[j] = lse_b[row[j]];
         }
@@ -94,7 +96,7 @@ merge_attn_states_lse_kernel(uint16_t *v_out, float *lse_out,
                 const float ta = mw.use_a ? fa[i] * mw.wa : 0.f;
                 fo[i] = mw.use_b ? fmaf(fb[i], mw.wb, ta) : ta;
             }
-            store<VEC, STH>(v_out + static_cast<int64_t>(v) * VEC, narrow<DT, VEC>(fo));
+            store<UV, STH>(v_out + static_cast<int64_t>(v) * UV, narrow<DT, VEC>(fo));
             if (lse_out != nullptr && v == row[j] * nvec.d) lse_out[row[j]] = mw.lse;
         }
     }
@@ -114,6 +116,7 @@ merge_attn_states_lse_strided_kernel(uint16_t *v_out, float *lse_out,
                                      const uint16_t *v_b, const float *lse_b,
                                      uint32_t total_vecs, uint32_t row0, FastDiv nvec, FastDiv heads,
                                      MergeStrides st) {
+    constexpr int UV = VEC * Storage<DT>::UNITS;  // 16-bit units per vector
     const uint32_t base = blockIdx.x * (THREADS * UNROLL) + threadIdx.x;
     grid_dependency_wait();
     grid_launch_dependents();
@@ -122,12 +125,12 @@ merge_attn_states_lse_strided_kernel(uint16_t *v_out, float *lse_out,
         const uint32_t v = base + j * THREADS;
         if (v < total_vecs) {
             const uint32_t lrow = nvec.div(v);
-            const int64_t col = static_cast<int64_t>(v - lrow * nvec.d) * VEC;
+            const int64_t col = static_cast<int64_t>(v - lrow * nvec.d) * UV;
             const uint32_t row = row0 + lrow;  // rows of this launch start at row0
             const uint32_t t = heads.div(row);
             const uint32_t h = row - t * heads.d;
-            const Pack<VEC> a = load<VEC, Ld::Stream>(v_a + (t * st.va_t + h * st.va_h + col));
-            const Pack<VEC> b = load<VEC, Ld::Stream>(v_b + (t * st.vb_t + h * st.vb_h + col));
+            const Pack<UV> a = load<UV, Ld::Stream>(v_a + (t * st.va_t + h * st.va_h + col));
+            const Pack<UV> b = load<UV, Ld::Stream>(v_b + (t * st.vb_t + h * st.vb_h + col));
             const MergeWeights mw = merge_weights(lse_a[t * st.sa_t + h * st.sa_h], lse_b[t * st.sb_t + h * st.sb_h]);
             float fa[VEC], fb[VEC], fo[VEC];
             widen<DT, VEC>(a, fa);
@@ -137,7 +140,7 @@ merge_attn_states_lse_strided_kernel(uint16_t *v_out, float *lse_out,
                 const float ta = mw.use_a ? fa[i] * mw.wa : 0.f;
                 fo[i] = mw.use_b ? fmaf(fb[i], mw.wb, ta) : ta;
             }
-            store<VEC, St::Stream>(v_out + (t * st.vo_t + h * st.vo_h + col), narrow<DT, VEC>(fo));
+            store<UV, St::Stream>(v_out + (t * st.vo_t + h * st.vo_h + col), narrow<DT, VEC>(fo));
             if (lse_out != nullptr && col == 0) lse_out[t * st.so_t + h * st.so_h] = mw.lse;
         }
     }

@@ -47,26 +47,27 @@ __device__ __forceinline__ float2 silu_mul2(float2 a, float2 b) {
 
 // Flat indexing: vector v of the output covers out[row, col*VEC .. col*VEC+VEC) with
 // row = v / nvec, col = v % nvec, nvec = D / VEC.  A block handles THREADS*UNROLL consecutive vectors.
-// gate and up are addressed separately (row pitches in elements), which covers both the packed
+// gate and up are addressed separately (pointers and row pitches in 16-bit units), which covers both the packed
 // row [a | b] (up = gate + D, equal pitches) and two independent tensors.
 template <int DT, int VEC, int UNROLL, int THREADS, Ld LDH = Ld::StreamReadOnly, St STH = St::Stream>
 __global__ void __launch_bounds__(THREADS)
 silu_and_mul_kernel(uint16_t *__restrict__ out, const uint16_t *__restrict__ gate,
                     const uint16_t *__restrict__ up, uint32_t total_vecs, FastDiv nvec,
                     int64_t out_pitch, int64_t gate_pitch, int64_t up_pitch) {
+    constexpr int UV = VEC * Storage<DT>::UNITS;  // 16-bit units per vector
     const uint32_t base = blockIdx.x * (THREADS * UNROLL) + threadIdx.x;
     grid_dependency_wait();
     grid_launch_dependents();
-    Pack<VEC> a[UNROLL], b[UNROLL];
+    Pack<UV> a[UNROLL], b[UNROLL];
 #pragma unroll
     for (int j = 0; j < UNROLL; ++j) {
         const uint32_t v = base + j * THREADS;
         if (v < total_vecs) {
             const uint32_t row = nvec.div(v);
             const uint32_t col = v - row * nvec.d;
-            const int64_t c = static_cast<int64_t>(col) * VEC;
-            a[j] = load<VEC, LDH>(gate + (static_cast<int64_t>(row) * gate_pitch + c));
-            b[j] = load<VEC, LDH>(up + (static_cast<int64_t>(row) * up_pitch + c));
+            const int64_t c = static_cast<int64_t>(col) * UV;
+            a[j] = load<UV, LDH>(gate + (static_cast<int64_t>(row) * gate_pitch + c));
+            b[j] = load<UV, LDH>(up + (static_cast<int64_t>(row) * up_pitch + c));
         }
     }
 #pragma unroll
@@ -88,7 +89,7 @@ silu_and_mul_kernel(uint16_t *__restrict__ out, const uint16_t *__restrict__ gat
             }
             const uint32_t row = nvec.div(v);
             const uint32_t col = v - row * nvec.d;
-            store<VEC, STH>(out + (static_cast<int64_t>(row) * out_pitch + static_cast<int64_t>(col) * VEC),
+            store<UV, STH>(out + (static_cast<int64_t>(row) * out_pitch + static_cast<int64_t>(col) * UV),
                             narrow<DT, VEC>(fo));
         }
     }

@@ -20,6 +20,7 @@ namespace astra {
 template <int DT> struct Storage;
 
 template <> struct Storage<ASTRA_BF16> {
+    static constexpr int UNITS = 1;  // 16-bit units per element
     static __device__ __forceinline__ void widen2(uint32_t w, float &lo, float &hi) {
         lo = __uint_as_float(w << 16);
         hi = __uint_as_float(w & 0xffff0000u);
@@ -37,6 +38,7 @@ template <> struct Storage<ASTRA_BF16> {
 };
 
 template <> struct Storage<ASTRA_FP16> {
+    static constexpr int UNITS = 1;
     static __device__ __forceinline__ void widen2(uint32_t w, float &lo, float &hi) {
         float2 f = __half22float2(*reinterpret_cast<__half2 *>(&w));
         lo = f.x;
@@ -54,9 +56,15 @@ template <> struct Storage<ASTRA_FP16> {
     }
 };
 
+// binary32 storage: an element is two 16-bit units (one 32-bit word) and needs no conversion.
+template <> struct Storage<ASTRA_FP32> {
+    static constexpr int UNITS = 2;
+};
+
 // ---------------------------------------------------------------------------------------------
-// A group of VEC consecutive 16-bit elements moved with one global access of 2*VEC bytes.
-// VEC = 1 is the scalar fallback for odd widths or 2-byte-aligned pointers.
+// A group of N consecutive 16-bit units moved with one global access of 2*N bytes (all tensors are
+// addressed in 16-bit units; an element of storage type DT is Storage<DT>::UNITS of them).
+// N = 1 is the scalar fallback for odd widths or 2-byte-aligned pointers of the 16-bit types.
 // ---------------------------------------------------------------------------------------------
 enum class Ld { Stream, StreamReadOnly, Keep };  // once-touched / once-touched and never written / reused (weights)
 enum class St { Stream, Default };
@@ -160,9 +168,13 @@ template <int VEC, St HINT> __device__ __forceinline__ void store(uint16_t *p, c
     }
 }
 
-// Pack<VEC> <-> VEC floats.
-template <int DT, int VEC> __device__ __forceinline__ void widen(const Pack<VEC> &v, float (&f)[VEC]) {
-    if constexpr (VEC == 1) {
+// Pack of VEC elements of storage type DT  <->  VEC floats.
+template <int DT, int VEC>
+__device__ __forceinline__ void widen(const Pack<VEC * Storage<DT>::UNITS> &v, float (&f)[VEC]) {
+    if constexpr (DT == ASTRA_FP32) {
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) f[i] = __uint_as_float(v.w[i]);
+    } else if constexpr (VEC == 1) {
         f[0] = Storage<DT>::widen1(static_cast<uint16_t>(v.w[0]));
     } else {
 #pragma unroll
@@ -170,9 +182,13 @@ template <int DT, int VEC> __device__ __forceinline__ void widen(const Pack<VEC>
     }
 }
 
-template <int DT, int VEC> __device__ __forceinline__ Pack<VEC> narrow(const float (&f)[VEC]) {
-    Pack<VEC> v;
-    if constexpr (VEC == 1) {
+template <int DT, int VEC>
+__device__ __forceinline__ Pack<VEC * Storage<DT>::UNITS> narrow(const float (&f)[VEC]) {
+    Pack<VEC * Storage<DT>::UNITS> v;
+    if constexpr (DT == ASTRA_FP32) {
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) v.w[i] = __float_as_uint(f[i]);
+    } else if constexpr (VEC == 1) {
         v.w[0] = Storage<DT>::narrow1(f[0]);
     } else {
 #pragma unroll

@@ -16,9 +16,11 @@ import torch
 
 BF16 = 0
 FP16 = 1
+FP32 = 2
 
-_TORCH_DTYPE = {BF16: torch.bfloat16, FP16: torch.float16}
-DTYPE_NAME = {BF16: "bf16", FP16: "fp16"}
+_TORCH_DTYPE = {BF16: torch.bfloat16, FP16: torch.float16, FP32: torch.float32}
+DTYPE_NAME = {BF16: "bf16", FP16: "fp16", FP32: "fp32"}
+ELEM_BYTES = {BF16: 2, FP16: 2, FP32: 4}
 
 
 def torch_dtype(dtype: int) -> torch.dtype:
@@ -26,13 +28,18 @@ def torch_dtype(dtype: int) -> torch.dtype:
 
 
 def bits(t: torch.Tensor) -> np.ndarray:
-    """The 16-bit storage patterns of a bf16/fp16 host tensor, as a uint16 numpy array."""
-    assert t.dtype in (torch.bfloat16, torch.float16) and t.device.type == "cpu"
+    """The storage patterns of a host tensor: uint16 for bf16/fp16, uint32 for fp32."""
+    assert t.device.type == "cpu"
+    if t.dtype == torch.float32:
+        return t.contiguous().view(torch.int32).numpy().view(np.uint32)
+    assert t.dtype in (torch.bfloat16, torch.float16)
     return t.contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
 def from_bits(a: np.ndarray, dtype: int) -> torch.Tensor:
     """Inverse of :func:`bits`."""
+    if dtype == FP32:
+        return torch.from_numpy(np.ascontiguousarray(a).view(np.int32)).view(torch.float32)
     return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(_TORCH_DTYPE[dtype])
 
 

@@ -7,6 +7,11 @@ Gates (oracle values are fp64; GPU values are the exact values of its 16-bit out
   - fp16 outputs: |gpu - oracle| <= max(1e-3, 2 * ulp_fp16(|oracle|)), ulp_fp16(v) = 2^(floor(log2 v) - 10)
     (floored at 2^-24).  The plain 1e-3 cannot hold above |y| = 4, where half an fp16 ulp already
     exceeds it; the count of elements beyond the literal 1e-3 is returned for reporting.
+  - fp32 outputs (storage without rounding, arithmetic with the GPU's approximate exp2,
+    reciprocal and rsqrt, each good to about 2 ulp): |gpu - oracle| <= 16 * ulp_fp32(|oracle|) for
+    rmsnorm and merge (plus the merge floor below).  For silu the exponent's argument |a|*log2(e)/2
+    is rounded to binary32 before exp2, which costs |a| * 2^-24 relative: the gate there is
+    (16 + 2*|a|) ulp, passed in through `extra`.
   - merge values: the blend a*Va + b*Vb can cancel, so the binary32 accumulation floor
     2^-22 * (|a*Va| + |b*Vb|) is added to the gate.
   - merged score: |gpu - oracle| <= 1e-5; -inf must be -inf.
@@ -15,9 +20,10 @@ from __future__ import annotations
 
 import numpy as np
 
-BF16, FP16 = 0, 1
-_FRAC = {BF16: 7, FP16: 10}
-_EMIN = {BF16: -126, FP16: -14}
+BF16, FP16, FP32 = 0, 1, 2
+_FRAC = {BF16: 7, FP16: 10, FP32: 23}
+_EMIN = {BF16: -126, FP16: -14, FP32: -126}
+_GATE_ULPS = {BF16: 2.0, FP16: 2.0, FP32: 16.0}
 
 
 def ulp(v: np.ndarray, dtype: int) -> np.ndarray:
@@ -33,7 +39,7 @@ def ulp(v: np.ndarray, dtype: int) -> np.ndarray:
 
 
 def value_gate(oracle: np.ndarray, dtype: int, extra: np.ndarray | float = 0.0) -> np.ndarray:
-    tol = 2.0 * ulp(oracle, dtype)
+    tol = _GATE_ULPS[dtype] * ulp(oracle, dtype)
     if dtype == FP16:
         tol = np.maximum(tol, 1e-3)
     tol = np.where(oracle == 0.0, 0.0, tol)

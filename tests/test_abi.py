@@ -95,7 +95,7 @@ def test_silu_argument_errors(lib):
     f = lib.astra_silu_and_mul
     assert f(None, A, 1, 8, 0, None) == binding.ASTRA_ERR_NULL_POINTER
     assert f(A, None, 1, 8, 0, None) == binding.ASTRA_ERR_NULL_POINTER
-    assert f(A, 2 * A, 1, 8, 2, None) == binding.ASTRA_ERR_BAD_DTYPE
+    assert f(A, 2 * A, 1, 8, 9, None) == binding.ASTRA_ERR_BAD_DTYPE
     assert f(A, 2 * A, -5, 8, 0, None) == binding.ASTRA_ERR_BAD_SHAPE
     assert f(A, 2 * A, 1, 0, 0, None) == binding.ASTRA_ERR_BAD_SHAPE
     assert f(A, 2 * A, 1, 2 ** 30, 0, None) == binding.ASTRA_ERR_BAD_SHAPE
@@ -216,3 +216,18 @@ def test_interleaved_slices_of_one_buffer_are_not_overlap(lib):
     assert f(x, A + 2 * (pitch - 4), x, A + 2 * (pitch - 4), w, 4, H, pitch, pitch, pitch, pitch, 1e-6, 0, None) \
         == binding.ASTRA_ERR_OVERLAP
     assert r  # the accepting direction is covered by the GPU tests (slices of one buffer)
+
+
+def test_fp32_storage_needs_four_byte_alignment(lib):
+    FP32 = binding.ASTRA_FP32
+    assert FP32 == 2
+    # 2-byte-aligned pointers are fine for the 16-bit types and misaligned for fp32
+    assert lib.astra_silu_and_mul(A + 2, 2 * A, 0, 8, 0, None) == binding.ASTRA_OK
+    assert lib.astra_silu_and_mul(A + 2, 2 * A, 1, 8, FP32, None) == binding.ASTRA_ERR_MISALIGNED
+    assert lib.astra_fused_add_rmsnorm(A, 2 * A + 2, 3 * A, 1, 8, 1e-6, FP32, None) == binding.ASTRA_ERR_MISALIGNED
+    assert lib.astra_merge_attn_states_lse(A, 2 * A, 3 * A + 2, 4 * A, 5 * A, 6 * A, 1, 2, 8, FP32, None) \
+        == binding.ASTRA_ERR_MISALIGNED
+    # overlap is judged in bytes of the storage type: [A, A+32) and [A+16, ...) overlap for fp32 rows of 8
+    assert lib.astra_fused_add_rmsnorm(A, A + 16, 3 * A, 1, 8, 1e-6, FP32, None) == binding.ASTRA_ERR_OVERLAP
+    assert lib.astra_silu_and_mul(A + 40, A, 1, 8, FP32, None) == binding.ASTRA_ERR_OVERLAP   # inside the up half
+    assert lib.astra_silu_and_mul(A, 2 * A, 0, 8, FP32, None) == binding.ASTRA_OK

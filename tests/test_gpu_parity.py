@@ -8,7 +8,7 @@ import torch
 import oracle
 import paper_2509_07506_b200 as astra
 from paper_2509_07506_b200 import workloads as wl
-from parity import check_lse, check_values
+from parity import check_lse, check_values, ulp
 
 pytestmark = pytest.mark.gpu
 
@@ -85,7 +85,10 @@ def run_silu(inp: wl.SiluInputs, rows=None, offset=0):
         return {}
     idx = torch.from_numpy(rows)
     want = oracle.silu_and_mul(wl.bits(inp.input[idx]), inp.dtype, nthreads=NCPU)
-    return check_values(f64(out[idx]), want, inp.dtype, what=f"silu {tuple(inp.input.shape)}")
+    extra = 0.0
+    if inp.dtype == wl.FP32:  # the exponent's argument is rounded to binary32: |a| * 2^-24 relative
+        extra = 2.0 * np.abs(f64(inp.input[idx][:, :D])) * ulp(np.where(want == 0, 1.0, want), inp.dtype) * (want != 0)
+    return check_values(f64(out[idx]), want, inp.dtype, extra=extra, what=f"silu {tuple(inp.input.shape)}")
 
 
 def run_merge(inp: wl.MergeInputs, tokens=None, offset=0, in_place=None, with_lse=True):
@@ -123,6 +126,8 @@ def run_merge(inp: wl.MergeInputs, tokens=None, offset=0, in_place=None, with_ls
     va = torch.nan_to_num(inp.v_a[idx].to(torch.float64), nan=0.0, posinf=0.0, neginf=0.0)
     vb = torch.nan_to_num(inp.v_b[idx].to(torch.float64), nan=0.0, posinf=0.0, neginf=0.0)
     floor = 2.0 ** -22 * ((w[..., 0:1] * va).abs() + (w[..., 1:2] * vb).abs()).numpy()
+    if inp.dtype == wl.FP32:  # the weights themselves carry a few binary32 ulp
+        floor = 4.0 * floor
     stats = check_values(f64(v[idx]), ov, inp.dtype, extra=floor, what=f"merge {tuple(inp.v_a.shape)}")
     if with_lse:
         stats["max_lse_err"] = check_lse(s[idx].numpy(), os_, what=f"merge lse {tuple(inp.v_a.shape)}")

@@ -22,16 +22,16 @@ MUTATIONS = [
     ("rmsnorm: eps dropped",
      "sqrt(sum_sq / (double)H + (double)eps)", "sqrt(sum_sq / (double)H)"),
     ("rmsnorm: weight indexed from the other end",
-     "/ denom * widen(w[j], f)", "/ denom * widen(w[H - 1 - j], f)"),
+     "/ denom * load_value(w, j, dtype, f)", "/ denom * load_value(w, H - 1 - j, dtype, f)"),
     ("rmsnorm: weight dropped",
-     "/ denom * widen(w[j], f)", "/ denom"),
+     "/ denom * load_value(w, j, dtype, f)", "/ denom"),
     ("rmsnorm: norm taken from the stored residual instead of the binary32 sum",
-     "double s = (double)(float)s_exact;                  /* binary32 add    */",
-     "double s = widen(round_to_storage((double)(float)s_exact, f), f);"),
+     "double s = (double)add_binary32(xv, rv, dtype);",
+     "double s = widen(round_to_storage((double)add_binary32(xv, rv, dtype), f), f);"),
     ("rmsnorm: x - r instead of x + r (both loops)",
-     "widen(xt[j], f) + widen(rt[j], f)", "widen(xt[j], f) - widen(rt[j], f)"),
+     "return (float)(a + b);", "return (float)(a - b);"),
     ("rmsnorm: residual gets x only",
-     "float s32 = (float)s_exact;", "float s32 = (float)widen(xt[j], f);"),
+     "float s32 = add_binary32(xv, rv, dtype);", "float s32 = (float)xv;"),
     ("rmsnorm: divides by the mean square instead of its root",
      "double denom = sqrt(", "double denom = ("),
     ("silu: e^{+z} in the denominator",
@@ -39,15 +39,15 @@ MUTATIONS = [
     ("silu: sigmoid instead of SiLU (z dropped)",
      "return z / (1.0 + exp(-z));", "return 1.0 / (1.0 + exp(-z));"),
     ("silu: gate and up halves swapped",
-     "double a = widen(row[i], f);\n            double b = widen(row[D + i], f);",
-     "double a = widen(row[D + i], f);\n            double b = widen(row[i], f);"),
+     "double a = load_value(input, row + i, dtype, f);\n            double b = load_value(input, row + D + i, dtype, f);",
+     "double a = load_value(input, row + D + i, dtype, f);\n            double b = load_value(input, row + i, dtype, f);"),
     ("silu: multiplication by b dropped",
      "out[t * D + i] = silu(a) * b;", "out[t * D + i] = silu(a);"),
     ("silu: row pitch D instead of 2D",
-     "const uint16_t *row = input + t * 2 * D;", "const uint16_t *row = input + t * D;"),
+     "const int64_t row = t * 2 * D;", "const int64_t row = t * D;"),
     ("merge: weights applied to the wrong states",
-     "if (wa != 0.0) num += wa * widen(va[d], f);\n            if (wb != 0.0) num += wb * widen(vb[d], f);",
-     "if (wa != 0.0) num += wa * widen(vb[d], f);\n            if (wb != 0.0) num += wb * widen(va[d], f);"),
+     "if (wa != 0.0) num += wa * load_value(v_a, base + d, dtype, f);\n            if (wb != 0.0) num += wb * load_value(v_b, base + d, dtype, f);",
+     "if (wa != 0.0) num += wa * load_value(v_b, base + d, dtype, f);\n            if (wb != 0.0) num += wb * load_value(v_a, base + d, dtype, f);"),
     ("merge: normalisation dropped",
      "vo[d] = num / denom;", "vo[d] = num;"),
     ("merge: max dropped from the merged score",
@@ -59,11 +59,15 @@ MUTATIONS = [
     ("merge: both-empty case not handled",
      "if (sa == -INFINITY && sb == -INFINITY) {", "if (0) {"),
     ("merge: zero-weight side multiplied instead of skipped",
-     "if (wb != 0.0) num += wb * widen(vb[d], f);", "num += wb * widen(vb[d], f);"),
+     "if (wb != 0.0) num += wb * load_value(v_b, base + d, dtype, f);", "num += wb * load_value(v_b, base + d, dtype, f);"),
     ("merge: scores indexed per token instead of per (token, head)",
      "double sb = (double)lse_b[th];", "double sb = (double)lse_b[th / Hh];"),
     ("storage: fp16 exponent bias off by one",
      "f.frac_bits = 10; f.exp_bits = 5; f.bias = 15;", "f.frac_bits = 10; f.exp_bits = 5; f.bias = 16;"),
+    ("storage: fp32 elements read at a 2-byte pitch",
+     "memcpy(&v, (const unsigned char *)base + 4 * i, 4);", "memcpy(&v, (const unsigned char *)base + 2 * i, 4);"),
+    ("storage: fp32 addition carried out in double and rounded afterwards twice (to bf16 precision)",
+     "volatile float s = fa + fb;", "volatile float s = (float)widen(round_to_storage((double)(fa + fb), format_of(0)), format_of(0));"),
     ("storage: bf16 read with 8 fraction bits",
      "f.frac_bits = 7;  f.exp_bits = 8; f.bias = 127;", "f.frac_bits = 8;  f.exp_bits = 8; f.bias = 127;"),
     ("storage: truncation instead of round-to-nearest-even",

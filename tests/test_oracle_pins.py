@@ -17,9 +17,10 @@ import torch
 import oracle
 from paper_2509_07506_b200 import workloads as wl
 
-BF16, FP16 = wl.BF16, wl.FP16
-DTYPES = [BF16, FP16]
-TD = {BF16: torch.bfloat16, FP16: torch.float16}
+BF16, FP16, FP32 = wl.BF16, wl.FP16, wl.FP32
+DTYPES = [BF16, FP16]                # the 16-bit storage formats (helpers that take 16-bit patterns)
+VALUE_DTYPES = [BF16, FP16, FP32]    # every storage type of the three operations
+TD = {BF16: torch.bfloat16, FP16: torch.float16, FP32: torch.float32}
 
 
 def golden():
@@ -45,7 +46,8 @@ def enc(values, dtype):
 
 def dec(bits_arr, dtype):
     """Exact float64 values of storage patterns, via torch's cast (independent of the oracle)."""
-    return wl.from_bits(np.asarray(bits_arr, dtype=np.uint16), dtype).to(torch.float64).numpy()
+    pat = np.uint32 if dtype == FP32 else np.uint16
+    return wl.from_bits(np.asarray(bits_arr, dtype=pat), dtype).to(torch.float64).numpy()
 
 
 # ---------------------------------------------------------------------------------------
@@ -184,7 +186,7 @@ def test_residual_sum_bf16_against_integer_adder():
     assert np.array_equal(r_out.ravel(), want)
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
 def test_residual_sum_matches_torch_float_add(dtype):
     """Library pin: torch adds in binary32 and casts once to the storage dtype."""
     inp = wl.rmsnorm_inputs(64, 515, dtype, seed=77)
@@ -197,7 +199,7 @@ def test_residual_sum_matches_torch_float_add(dtype):
 # fused_add_rmsnorm  (Table 1, Kernel 2)
 # ---------------------------------------------------------------------------------------
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
 def test_rmsnorm_hand_value_3_4(dtype):
     # x + r = [3, 4] split unevenly between x and r; eps = 0; weights [2, 0.5]
     x = enc([[1.0, 5.0]], dtype); r = enc([[2.0, -1.0]], dtype); w = enc([2.0, 0.5], dtype)
@@ -208,7 +210,7 @@ def test_rmsnorm_hand_value_3_4(dtype):
     assert np.array_equal(r_out, enc([[3.0, 4.0]], dtype))
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
 @pytest.mark.parametrize("c", [0.5, -2.0, 3.0])
 def test_rmsnorm_constant_row_closed_form(dtype, c):
     H = 37
@@ -221,12 +223,13 @@ def test_rmsnorm_constant_row_closed_form(dtype, c):
     eps_f = float(np.float32(eps))
     want = c / math.sqrt(c * c + eps_f) * wt.to(torch.float64).numpy()
     np.testing.assert_allclose(y[0], want, rtol=1e-14)
-    # for eps << c^2 the row normalises to sign(c) * w after storage rounding
-    stored = wl.bits(torch.from_numpy(y[0]).to(TD[dtype]))
-    assert np.array_equal(stored, wl.bits((math.copysign(1.0, c) * wt.to(torch.float64)).to(TD[dtype])))
+    # for eps << c^2 the row normalises to sign(c) * w after rounding to a 16-bit storage type
+    if dtype != FP32:
+        stored = wl.bits(torch.from_numpy(y[0]).to(TD[dtype]))
+        assert np.array_equal(stored, wl.bits((math.copysign(1.0, c) * wt.to(torch.float64)).to(TD[dtype])))
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
 def test_rmsnorm_zero_row_is_zero(dtype):
     x = enc([[0.0] * 9, [1.0] * 9], dtype); r = enc([[0.0] * 9, [-1.0] * 9], dtype)
     w = enc([1.5] * 9, dtype)
@@ -235,7 +238,7 @@ def test_rmsnorm_zero_row_is_zero(dtype):
     assert np.all(r_out == 0)
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
 @pytest.mark.parametrize("eps", [1e-6, 1e-5, 0.5])
 def test_rmsnorm_mean_square_invariant_and_eps_placement(dtype, eps):
     """mean_j (y_j / w_j)^2 = m / (m + eps): holds only with eps inside the root, added to the mean."""
@@ -255,7 +258,7 @@ def test_rmsnorm_power_of_two_scaling_invariance():
     np.testing.assert_allclose(y2, y1, rtol=1e-15)
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
 def test_rmsnorm_reduces_to_library_rms_norm(dtype):
     """r = 0, w = 1 is plain RMSNorm; the general case is rms_norm of the binary32 sum."""
     inp = wl.rmsnorm_inputs(7, 200, dtype, eps=1e-5, seed=9)
@@ -297,7 +300,7 @@ def test_rmsnorm_rows_are_independent_and_weight_indexed_by_column():
 # silu_and_mul  (Table 1, Kernel 3)
 # ---------------------------------------------------------------------------------------
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
 def test_silu_hand_values_and_layout(dtype):
     # row = [gate | up]; D = 3
     row = enc([[1.0, -1.0, 2.0, 1.0, 1.0, 1.0]], dtype)
@@ -312,7 +315,7 @@ def test_silu_hand_values_and_layout(dtype):
     assert out[0, 0] == pytest.approx(2 * GOLD["sigmoid_1"], rel=1e-15)
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
 def test_silu_zero_odd_part_and_limits(dtype):
     a = [0.0, -0.0, 0.37, 1.5, 7.25, 30.0, 60.0]
     D = len(a)
@@ -332,7 +335,7 @@ def test_silu_zero_odd_part_and_limits(dtype):
     np.testing.assert_allclose(out, -pos, rtol=0, atol=0)
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
 def test_silu_matches_library_silu(dtype):
     inp = wl.silu_inputs(9, 77, dtype, std=2.0, seed=5)
     out = oracle.silu_and_mul(wl.bits(inp.input), dtype)
@@ -360,7 +363,7 @@ def _merge(va, sa, vb, sb, dtype=BF16):
     return v, s
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
 def test_merge_equal_scores_give_mean_and_ln2(dtype):
     va = [[[1.0, -2.0, 0.5, 3.0]]]; vb = [[[3.0, 2.0, 0.25, -3.0]]]
     for s in (0.0, 7.5, -40.0, 80.0):
@@ -377,7 +380,7 @@ def test_merge_hand_weight_three_quarters():
     assert so[0, 0] == pytest.approx(math.log(4.0), rel=2e-7)
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
 def test_merge_neg_inf_returns_other_state(dtype):
     ninf = float("-inf")
     va = [[[1.5, -2.0, 0.0, 7.0]]]; vb = [[[9.0, 9.0, -9.0, 1.0]]]
@@ -402,7 +405,7 @@ def test_merge_out_of_domain_scores_give_nan():
     assert np.isnan(v).all() and np.isnan(s).all()
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
 def test_merge_symmetry_shift_and_bounds(dtype):
     inp = wl.merge_inputs(11, 3, 20, dtype, seed=13, neg_inf_frac=0.0, forced_both_neg_inf=0)
     va, vb = wl.bits(inp.v_a), wl.bits(inp.v_b)
@@ -419,7 +422,7 @@ def test_merge_symmetry_shift_and_bounds(dtype):
     assert np.all(s >= m) and np.all(s <= m + GOLD["ln_2"] + 1e-15)
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
 def test_merge_matches_library_softmax_and_logaddexp(dtype):
     inp = wl.merge_inputs(9, 5, 24, dtype, seed=31)
     v, s = oracle.merge_attn_states_lse(wl.bits(inp.v_a), inp.lse_a.numpy(), wl.bits(inp.v_b),
@@ -481,7 +484,7 @@ def _D(v):
     return decimal.Decimal(float(v))
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
 def test_tiny_shapes_against_50_digit_arithmetic(dtype):
     decimal.getcontext().prec = 50
     for T in (1, 2, 3):
