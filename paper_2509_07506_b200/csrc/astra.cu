@@ -92,6 +92,33 @@ inline void launch(void (*kernel)(KArgs...), unsigned grid, unsigned block, cuda
 #ifndef ASTRA_MAX_ROWS_PER_LAUNCH
 #define ASTRA_MAX_ROWS_PER_LAUNCH 2147483647
 #endif
+// Preferred upper bound on the block size of the cluster kernel (more, smaller blocks per row are
+// chosen while the cluster size allows it).
+#ifndef ASTRA_CLUSTER_PREFERRED_THREADS
+#define ASTRA_CLUSTER_PREFERRED_THREADS 512
+#endif
+// The same, for a kernel whose consecutive groups of `cluster` blocks form thread-block clusters
+// (distributed shared memory between the blocks of a group).
+template <typename... KArgs, typename... Args>
+inline void launch_clustered(void (*kernel)(KArgs...), unsigned grid, unsigned block, unsigned cluster,
+                             cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = cluster;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 constexpr int64_t kMaxVecsPerLaunch = ASTRA_MAX_VECS_PER_LAUNCH;
 constexpr int64_t kInt64Max = 9223372036854775807ll;
 
@@ -269,9 +296,9 @@ inline bool rows_disjoint(int64_t T, int64_t Hh, int64_t W, int64_t st, int64_t 
 // ---------------------------------------------------------------------------------------------
 constexpr int kMaxGridX = ASTRA_MAX_ROWS_PER_LAUNCH;
 
-// Most 16-bit units of a row one thread keeps in registers: 64 with vector accesses, 16 on the
+// Most 16-bit units of a row one thread keeps in registers: 64 with vector accesses, 8 on the
 // scalar path (each element then also costs three separate packed-input registers).
-constexpr int rmsnorm_max_units_per_thread(int uvec) { return uvec == 1 ? 16 : 64; }
+constexpr int rmsnorm_max_units_per_thread(int uvec) { return uvec == 1 ? 8 : 64; }
 
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
@@ -299,21 +326,45 @@ void launch_rmsnorm(RmsnormOperands op, const uint16_t *w, int64_t T, int H, flo
     const float inv_H = 1.0f / static_cast<float>(H);
     // start at 16 units per thread; widen the per-thread share only if the row needs more threads
     // than that share allows, narrow it if the block would fall under 128 threads
-    int vpt = 16 / UVEC < 1 ? 1 : 16 / UVEC;
+    int vpt = UVEC == 1 ? 8 : 16 / UVEC;
     auto threads_for = [&](int v) { return round_up((nvec + v - 1) / v, 32); };
     while (vpt < kMaxVpt && threads_for(vpt) > rmsnorm_reg_max_threads(UVEC * vpt)) vpt <<= 1;
     while (vpt > 1 && threads_for(vpt) < 128) vpt >>= 1;
     const int threads = threads_for(vpt);
     const bool fits = threads <= rmsnorm_reg_max_threads(UVEC * vpt);
-    for (int64_t t0 = 0; t0 < T; t0 += kMaxGridX) {
-        const unsigned rows = static_cast<unsigned>(T - t0 < kMaxGridX ? T - t0 : kMaxGridX);
+    // Wider rows: share the row among a cluster of 2, 4 or 8 blocks (the portable maximum), each
+    // holding 16 units per thread; only beyond 8 x 1024 x 16 units per row fall back to two sweeps.
+    constexpr int kClusterVpt = (16 / UVEC < 1 ? 1 : 16 / UVEC);
+    int cluster = 0, cluster_threads = 0;
+    if (!fits && UVEC >= 4) {  // vector paths only; scalar and 4-byte rows take the two-sweep kernel
+        for (int c = 2; c <= 8; c <<= 1) {
+            const int chunk = (nvec + c - 1) / c;
+            const int th = round_up((chunk + kClusterVpt - 1) / kClusterVpt, 32);
+            if (th > rmsnorm_reg_max_threads(UVEC * kClusterVpt)) continue;
+            if (cluster != 0 && cluster_threads <= ASTRA_CLUSTER_PREFERRED_THREADS) break;
+            cluster = c;
+            cluster_threads = th;
+        }
+    }
+    // two-sweep fallback: as few strided iterations per thread as 1024 threads allow, evenly filled
+    const int sweep_iters = (nvec + 1023) / 1024;
+    const int sweep_threads = round_up((nvec + sweep_iters - 1) / sweep_iters, 32);
+    const int64_t rows_per_launch = cluster ? kMaxGridX / cluster : kMaxGridX;
+    for (int64_t t0 = 0; t0 < T; t0 += rows_per_launch) {
+        const unsigned rows = static_cast<unsigned>(T - t0 < rows_per_launch ? T - t0 : rows_per_launch);
         RmsnormOperands o = op;
         o.x += t0 * op.x_pitch;
         o.r += t0 * op.r_pitch;
         o.y += t0 * op.y_pitch;
         o.r_out += t0 * op.r_out_pitch;
+        if (cluster) {
+            if constexpr (UVEC >= 4)
+                launch_clustered(fused_add_rmsnorm_cluster_kernel<DT, VEC, kClusterVpt>, rows * cluster,
+                                 cluster_threads, cluster, stream, o, w, H, eps, inv_H);
+            continue;
+        }
         if (!fits) {
-            launch(fused_add_rmsnorm_twopass_kernel<DT, VEC>, rows, 1024, stream, o, w, H, eps, inv_H);
+            launch(fused_add_rmsnorm_twopass_kernel<DT, VEC>, rows, sweep_threads, stream, o, w, H, eps, inv_H);
             continue;
         }
         switch (vpt) {

@@ -10,6 +10,8 @@
 // before anything is consumed; the weight (an L2 hit) is fetched while the reduction completes.
 #pragma once
 
+#include <cooperative_groups.h>
+
 #include "vec.cuh"
 
 namespace astra {
@@ -58,7 +60,7 @@ __host__ __device__ constexpr int rmsnorm_reg_max_threads(int units_per_thread) 
 // four-vector form (8-byte accesses, e.g. H = 4100) spills three registers under the cap and still
 // measured fastest; with eight or sixteen narrower vectors the spills grow, so no cap there.
 template <int DT, int VEC, int VPT, Ld LDH = Ld::Stream, St STH = St::Stream, bool EARLY_W = false,
-          int MINB = ((VEC * VPT * Storage<DT>::UNITS <= 16 && VPT <= 4) ? 2 : 1)>
+          int MINB = ((VEC * VPT * Storage<DT>::UNITS <= 16 && VPT <= 4 && VEC * Storage<DT>::UNITS >= 4) ? 2 : 1)>
 __global__ void __launch_bounds__(rmsnorm_reg_max_threads(VEC * VPT * Storage<DT>::UNITS), MINB)
 fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ weight,
                              int H, float eps, float inv_H) {
@@ -128,6 +130,89 @@ fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ we
 #pragma unroll
             for (int k = 0; k < VEC; ++k) fy[k] = s[i][k] * rstd * fw[k];
             store<UV, STH>(yr + v * UV, narrow<DT, VEC>(fy));
+        }
+    }
+}
+
+// Rows too wide for one block's registers: a thread-block cluster owns the row.  Each block keeps
+// its contiguous share of the row in registers exactly as above and reduces it; the per-block
+// partial sums are then exchanged through distributed shared memory (every block reads every
+// partial, in rank order, so all blocks form the same total bit for bit), and each block finishes
+// its share.  The row still makes one trip through HBM.  The two cluster barriers are hardware
+// barriers that every thread of every block reaches unconditionally (blocks without work included):
+// the first publishes the partials, the second keeps each block's shared memory alive until all its
+// peers have read it.
+template <int DT, int VEC, int VPT, int MINB = ((VEC * VPT * Storage<DT>::UNITS <= 16 && VPT <= 2) ? 2 : 1)>
+__global__ void __launch_bounds__(rmsnorm_reg_max_threads(VEC * VPT * Storage<DT>::UNITS), MINB)
+fused_add_rmsnorm_cluster_kernel(RmsnormOperands op, const uint16_t *__restrict__ weight,
+                                 int H, float eps, float inv_H) {
+    namespace cg = cooperative_groups;
+    constexpr int UV = VEC * Storage<DT>::UNITS;
+    __shared__ float slots[kMaxWarps];
+    __shared__ float block_partial;
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned nblocks = cluster.num_blocks();
+    const unsigned rank = cluster.block_rank();
+    const int nvec = H / VEC;
+    const int chunk = (nvec + nblocks - 1) / nblocks;  // vectors per block (the last may hold fewer)
+    const int first = rank * chunk;
+    const int count = max(0, min(chunk, nvec - first));
+    const int64_t row = blockIdx.x / nblocks;
+    const uint16_t *xr = op.x + row * op.x_pitch + static_cast<int64_t>(first) * UV;
+    const uint16_t *rr = op.r + row * op.r_pitch + static_cast<int64_t>(first) * UV;
+    uint16_t *yr = op.y + row * op.y_pitch + static_cast<int64_t>(first) * UV;
+    uint16_t *ror = op.r_out + row * op.r_out_pitch + static_cast<int64_t>(first) * UV;
+    const uint16_t *wr = weight + static_cast<int64_t>(first) * UV;
+    grid_dependency_wait();
+    grid_launch_dependents();
+
+    Pack<UV> px[VPT], pr[VPT], pw[VPT];
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int v = threadIdx.x + i * blockDim.x;
+        if (v < count) {
+            px[i] = load<UV, Ld::Stream>(xr + v * UV);
+            pr[i] = load<UV, Ld::Stream>(rr + v * UV);
+        }
+    }
+    float s[VPT][VEC];
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int v = threadIdx.x + i * blockDim.x;
+        if (v < count) {
+            float fx[VEC], fr[VEC];
+            widen<DT, VEC>(px[i], fx);
+            widen<DT, VEC>(pr[i], fr);
+#pragma unroll
+            for (int k = 0; k < VEC; ++k) {
+                s[i][k] = fx[k] + fr[k];
+                acc = fmaf(s[i][k], s[i][k], acc);
+            }
+            store<UV, St::Stream>(ror + v * UV, narrow<DT, VEC>(s[i]));
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int v = threadIdx.x + i * blockDim.x;
+        if (v < count) pw[i] = load<UV, Ld::Keep>(wr + v * UV);
+    }
+    const float mine = block_sum(acc, slots);
+    if (threadIdx.x == 0) block_partial = mine;
+    cluster.sync();
+    float total = 0.f;
+    for (unsigned b = 0; b < nblocks; ++b) total += *cluster.map_shared_rank(&block_partial, b);
+    cluster.sync();
+    const float rstd = rsqrtf(fmaf(total, inv_H, eps));
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int v = threadIdx.x + i * blockDim.x;
+        if (v < count) {
+            float fw[VEC], fy[VEC];
+            widen<DT, VEC>(pw[i], fw);
+#pragma unroll
+            for (int k = 0; k < VEC; ++k) fy[k] = s[i][k] * rstd * fw[k];
+            store<UV, St::Stream>(yr + v * UV, narrow<DT, VEC>(fy));
         }
     }
 }

@@ -16,7 +16,7 @@ FP32 = wl.FP32
 
 
 @pytest.mark.parametrize("T,H", [(16, 4096), (64, 8192), (5, 4100), (5, 4098), (3, 250), (2, 33), (3, 1), (4, 5120),
-                                 (3, 11008), (2, 14336), (2, 40000)])
+                                 (3, 11008), (2, 14336), (2, 40000), (3, 8200), (2, 65536), (2, 70000)])
 def test_rmsnorm_fp32(T, H):
     run_rmsnorm(wl.rmsnorm_inputs(T, H, FP32, eps=1e-5, seed=H))
 

@@ -194,8 +194,10 @@ def test_table4_shapes(dtype, kernel, shape):
 
 @pytest.mark.parametrize("dtype", [BF16, FP16])
 @pytest.mark.parametrize("H", [1, 2, 3, 7, 8, 9, 33, 250, 1000, 4100, 4101, 4098, 8190, 11008, 14336,
-                               32768, 32776, 40000, 65538])
+                               32768, 32776, 40000, 65538, 16392, 20500, 49152, 131072, 131080, 100000])
 def test_rmsnorm_widths(dtype, H):
+    # widths above 16384 exercise the cluster kernel (2, 4 or 8 blocks per row) and, beyond
+    # 131072 or with narrow vectors, the two-sweep kernel; T = 3 or 5 leaves a partial wave of clusters
     T = 3 if H > 20000 else 5
     run_rmsnorm(wl.rmsnorm_inputs(T, H, dtype, eps=1e-5, seed=H))
 

@@ -39,7 +39,7 @@ def untouched(buf, col0, width):
 
 @pytest.mark.parametrize("dtype", [BF16, FP16])
 @pytest.mark.parametrize("H,pitch,col0", [(4096, 4096 + 64, 0), (4096, 8192, 4096), (4100, 4100 + 12, 4),
-                                          (520, 777, 3), (8192, 8192 + 8, 8)])
+                                          (520, 777, 3), (8192, 8192 + 8, 8), (24576, 24576 + 64, 32), (40000, 40008, 8)])
 @pytest.mark.parametrize("in_place", [False, True])
 def test_rmsnorm_ex_pitched(dtype, H, pitch, col0, in_place):
     T = 37
