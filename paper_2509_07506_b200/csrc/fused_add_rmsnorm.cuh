@@ -140,8 +140,9 @@ fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ we
 // partial, in rank order, so all blocks form the same total bit for bit), and each block finishes
 // its share.  The row still makes one trip through HBM.  The two cluster barriers are hardware
 // barriers that every thread of every block reaches unconditionally (blocks without work included):
-// the first publishes the partials, the second keeps each block's shared memory alive until all its
-// peers have read it.
+// the first publishes the partials; the second, split into an arrive right after the partials are
+// read and a wait at the very end, keeps each block's shared memory alive until all its peers have
+// read it without stalling the final stores.
 template <int DT, int VEC, int VPT, int MINB = ((VEC * VPT * Storage<DT>::UNITS <= 16 && VPT <= 2) ? 2 : 1)>
 __global__ void __launch_bounds__(rmsnorm_reg_max_threads(VEC * VPT * Storage<DT>::UNITS), MINB)
 fused_add_rmsnorm_cluster_kernel(RmsnormOperands op, const uint16_t *__restrict__ weight,
@@ -202,7 +203,7 @@ fused_add_rmsnorm_cluster_kernel(RmsnormOperands op, const uint16_t *__restrict_
     cluster.sync();
     float total = 0.f;
     for (unsigned b = 0; b < nblocks; ++b) total += *cluster.map_shared_rank(&block_partial, b);
-    cluster.sync();
+    cluster.barrier_arrive();  // "I have read my peers' partials"; waited for just before exit
     const float rstd = rsqrtf(fmaf(total, inv_H, eps));
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
@@ -215,6 +216,7 @@ fused_add_rmsnorm_cluster_kernel(RmsnormOperands op, const uint16_t *__restrict_
             store<UV, St::Stream>(yr + v * UV, narrow<DT, VEC>(fy));
         }
     }
+    cluster.barrier_wait();  // no block leaves while a peer may still read its shared memory
 }
 
 // Any H: two sweeps over the row.  The first only reads (x, r) and accumulates the sum of squares;
