@@ -231,3 +231,32 @@ def test_fp32_storage_needs_four_byte_alignment(lib):
     assert lib.astra_fused_add_rmsnorm(A, A + 16, 3 * A, 1, 8, 1e-6, FP32, None) == binding.ASTRA_ERR_OVERLAP
     assert lib.astra_silu_and_mul(A + 40, A, 1, 8, FP32, None) == binding.ASTRA_ERR_OVERLAP   # inside the up half
     assert lib.astra_silu_and_mul(A, 2 * A, 0, 8, FP32, None) == binding.ASTRA_OK
+
+
+def test_headers_are_plain_c_and_link_from_c(tmp_path):
+    """The public headers compile as strict C99, and a C program linked against libastra.so can call
+    the error paths (nothing is launched)."""
+    import subprocess
+    astra_build.build()
+    src = tmp_path / "use_from_c.c"
+    src.write_text(r'''
+#include <stdio.h>
+#include "astra.h"
+#include "astra_ablation.h"
+int main(void) {
+    char buf[64] = {0};
+    astra_status_t s = astra_silu_and_mul(NULL, buf, 1, 8, ASTRA_BF16, NULL);
+    if (s != ASTRA_ERR_NULL_POINTER) return 1;
+    s = astra_fused_add_rmsnorm(buf, buf + 32, buf + 48, 0, 8, 1e-6f, ASTRA_FP32, NULL);
+    if (s != ASTRA_OK) return 2;
+    if (astra_status_string(ASTRA_ERR_OVERLAP)[0] == 0) return 3;
+    printf("%s\n", astra_status_string(s));
+    return 0;
+}
+''')
+    exe = tmp_path / "use_from_c"
+    libdir = os.path.dirname(astra_build.LIB_PATH)
+    subprocess.check_call(["gcc", "-std=c99", "-pedantic", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"),
+                           str(src), "-o", str(exe), "-L", libdir, "-lastra", f"-Wl,-rpath,{libdir}"])
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0 and out.stdout.strip() == "ok"
