@@ -244,7 +244,8 @@ def test_headers_are_plain_c_and_link_from_c(tmp_path):
 #include "astra.h"
 #include "astra_ablation.h"
 int main(void) {
-    char buf[64] = {0};
+    float store[16] = {0};
+    char *buf = (char *)store;  /* 4-byte aligned, as fp32 operands must be */
     astra_status_t s = astra_silu_and_mul(NULL, buf, 1, 8, ASTRA_BF16, NULL);
     if (s != ASTRA_ERR_NULL_POINTER) return 1;
     s = astra_fused_add_rmsnorm(buf, buf + 32, buf + 48, 0, 8, 1e-6f, ASTRA_FP32, NULL);
