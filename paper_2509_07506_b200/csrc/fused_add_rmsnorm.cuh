@@ -43,6 +43,46 @@ __device__ __forceinline__ float block_sum(float v, float *slots) {
     return t;
 }
 
+// s = x + r (one binary32 add per element) and the running sum of squares, two elements per
+// instruction with the packed binary32 forms of sm_100 where the vector has an even length (the
+// scalar accumulator serves one-element vectors).  Same roundings as the scalar forms.
+template <int VEC>
+__device__ __forceinline__ void add_and_square(const float (&x)[VEC], const float (&r)[VEC], float (&s)[VEC],
+                                               float &acc, float2 &acc2) {
+    if constexpr (VEC % 2 == 0) {
+#pragma unroll
+        for (int k = 0; k < VEC; k += 2) {
+            const float2 t = __fadd2_rn(make_float2(x[k], x[k + 1]), make_float2(r[k], r[k + 1]));
+            acc2 = __ffma2_rn(t, t, acc2);
+            s[k] = t.x;
+            s[k + 1] = t.y;
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) {
+            s[k] = x[k] + r[k];
+            acc = fmaf(s[k], s[k], acc);
+        }
+    }
+}
+
+// y = (s * rstd) * w, packed likewise.
+template <int VEC>
+__device__ __forceinline__ void scale(const float (&s)[VEC], float rstd, const float (&w)[VEC], float (&y)[VEC]) {
+    if constexpr (VEC % 2 == 0) {
+        const float2 r2 = make_float2(rstd, rstd);
+#pragma unroll
+        for (int k = 0; k < VEC; k += 2) {
+            const float2 t = __fmul2_rn(__fmul2_rn(make_float2(s[k], s[k + 1]), r2), make_float2(w[k], w[k + 1]));
+            y[k] = t.x;
+            y[k + 1] = t.y;
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) y[k] = s[k] * rstd * w[k];
+    }
+}
+
 // Largest block the register-resident kernel may be launched with, by vectors per thread: the
 // row's binary32 sums plus its packed inputs (counted in 16-bit units per thread) must fit the
 // register file.
@@ -57,8 +97,8 @@ __host__ __device__ constexpr int rmsnorm_reg_max_threads(int units_per_thread) 
 // the register allocation must allow; with 16 units per thread in at most four vectors MINB = 2
 // caps the kernel at 32 registers, i.e. full occupancy for every block size, which is worth 5 % at
 // [16384, 8192] and 27 % at [512, 14336] (896-thread blocks: two per SM instead of one).  The
-// four-vector form (8-byte accesses, e.g. H = 4100) spills three registers under the cap and still
-// measured fastest; with eight or sixteen narrower vectors the spills grow, so no cap there.
+// four-vector form (8-byte accesses, e.g. H = 4100) fits the cap too; with eight or sixteen narrower
+// vectors it would spill, so no cap there.
 template <int DT, int VEC, int VPT, Ld LDH = Ld::Stream, St STH = St::Stream, bool EARLY_W = false,
           int MINB = ((VEC * VPT * Storage<DT>::UNITS <= 16 && VPT <= 4 && VEC * Storage<DT>::UNITS >= 4) ? 2 : 1)>
 __global__ void __launch_bounds__(rmsnorm_reg_max_threads(VEC * VPT * Storage<DT>::UNITS), MINB)
@@ -95,6 +135,7 @@ fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ we
 
     float s[VPT][VEC];
     float acc = 0.f;
+    float2 acc2 = make_float2(0.f, 0.f);
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
         const int v = threadIdx.x + i * blockDim.x;
@@ -102,11 +143,7 @@ fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ we
             float fx[VEC], fr[VEC];
             widen<DT, VEC>(px[i], fx);
             widen<DT, VEC>(pr[i], fr);
-#pragma unroll
-            for (int k = 0; k < VEC; ++k) {
-                s[i][k] = fx[k] + fr[k];  // the one binary32 add
-                acc = fmaf(s[i][k], s[i][k], acc);
-            }
+            add_and_square(fx, fr, s[i], acc, acc2);  // the one binary32 add per element
             store<UV, STH>(ror + v * UV, narrow<DT, VEC>(s[i]));
         }
     }
@@ -118,7 +155,7 @@ fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ we
             if (v < nvec) pw[i] = load<UV, Ld::Keep>(weight + v * UV);
         }
     }
-    const float total = block_sum(acc, slots);
+    const float total = block_sum(acc + (acc2.x + acc2.y), slots);
     const float rstd = rsqrtf(fmaf(total, inv_H, eps));
 
 #pragma unroll
@@ -127,8 +164,7 @@ fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ we
         if (v < nvec) {
             float fw[VEC], fy[VEC];
             widen<DT, VEC>(pw[i], fw);
-#pragma unroll
-            for (int k = 0; k < VEC; ++k) fy[k] = s[i][k] * rstd * fw[k];
+            scale(s[i], rstd, fw, fy);
             store<UV, STH>(yr + v * UV, narrow<DT, VEC>(fy));
         }
     }
@@ -178,6 +214,7 @@ fused_add_rmsnorm_cluster_kernel(RmsnormOperands op, const uint16_t *__restrict_
     }
     float s[VPT][VEC];
     float acc = 0.f;
+    float2 acc2 = make_float2(0.f, 0.f);
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
         const int v = threadIdx.x + i * blockDim.x;
@@ -185,11 +222,7 @@ fused_add_rmsnorm_cluster_kernel(RmsnormOperands op, const uint16_t *__restrict_
             float fx[VEC], fr[VEC];
             widen<DT, VEC>(px[i], fx);
             widen<DT, VEC>(pr[i], fr);
-#pragma unroll
-            for (int k = 0; k < VEC; ++k) {
-                s[i][k] = fx[k] + fr[k];
-                acc = fmaf(s[i][k], s[i][k], acc);
-            }
+            add_and_square(fx, fr, s[i], acc, acc2);
             store<UV, St::Stream>(ror + v * UV, narrow<DT, VEC>(s[i]));
         }
     }
@@ -198,7 +231,7 @@ fused_add_rmsnorm_cluster_kernel(RmsnormOperands op, const uint16_t *__restrict_
         const int v = threadIdx.x + i * blockDim.x;
         if (v < count) pw[i] = load<UV, Ld::Keep>(wr + v * UV);
     }
-    const float mine = block_sum(acc, slots);
+    const float mine = block_sum(acc + (acc2.x + acc2.y), slots);
     if (threadIdx.x == 0) block_partial = mine;
     cluster.sync();
     float total = 0.f;
@@ -211,8 +244,7 @@ fused_add_rmsnorm_cluster_kernel(RmsnormOperands op, const uint16_t *__restrict_
         if (v < count) {
             float fw[VEC], fy[VEC];
             widen<DT, VEC>(pw[i], fw);
-#pragma unroll
-            for (int k = 0; k < VEC; ++k) fy[k] = s[i][k] * rstd * fw[k];
+            scale(s[i], rstd, fw, fy);
             store<UV, St::Stream>(yr + v * UV, narrow<DT, VEC>(fy));
         }
     }
