@@ -179,8 +179,8 @@ fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ we
 // the first publishes the partials; the second, split into an arrive right after the partials are
 // read and a wait at the very end, keeps each block's shared memory alive until all its peers have
 // read it without stalling the final stores.
-// (the register cap is kept for fp32 although that instantiation spills 48 bytes: without it the
-// lower occupancy costs 20 % at [2048, 14336] fp32)
+// (scalar arithmetic here: the packed forms cost the registers that keep this kernel at full
+// occupancy, which matters more: 5.4 against 4.5 TB/s at [2048, 14336] fp32)
 template <int DT, int VEC, int VPT, int MINB = ((VEC * VPT * Storage<DT>::UNITS <= 16 && VPT <= 2) ? 2 : 1)>
 __global__ void __launch_bounds__(rmsnorm_reg_max_threads(VEC * VPT * Storage<DT>::UNITS), MINB)
 fused_add_rmsnorm_cluster_kernel(RmsnormOperands op, const uint16_t *__restrict__ weight,
@@ -216,7 +216,6 @@ fused_add_rmsnorm_cluster_kernel(RmsnormOperands op, const uint16_t *__restrict_
     }
     float s[VPT][VEC];
     float acc = 0.f;
-    float2 acc2 = make_float2(0.f, 0.f);
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
         const int v = threadIdx.x + i * blockDim.x;
@@ -224,7 +223,11 @@ fused_add_rmsnorm_cluster_kernel(RmsnormOperands op, const uint16_t *__restrict_
             float fx[VEC], fr[VEC];
             widen<DT, VEC>(px[i], fx);
             widen<DT, VEC>(pr[i], fr);
-            add_and_square(fx, fr, s[i], acc, acc2);
+#pragma unroll
+            for (int k = 0; k < VEC; ++k) {
+                s[i][k] = fx[k] + fr[k];
+                acc = fmaf(s[i][k], s[i][k], acc);
+            }
             store<UV, St::Stream>(ror + v * UV, narrow<DT, VEC>(s[i]));
         }
     }
@@ -233,7 +236,7 @@ fused_add_rmsnorm_cluster_kernel(RmsnormOperands op, const uint16_t *__restrict_
         const int v = threadIdx.x + i * blockDim.x;
         if (v < count) pw[i] = load<UV, Ld::Keep>(wr + v * UV);
     }
-    const float mine = block_sum(acc + (acc2.x + acc2.y), slots);
+    const float mine = block_sum(acc, slots);
     if (threadIdx.x == 0) block_partial = mine;
     cluster.sync();
     float total = 0.f;
@@ -246,7 +249,8 @@ fused_add_rmsnorm_cluster_kernel(RmsnormOperands op, const uint16_t *__restrict_
         if (v < count) {
             float fw[VEC], fy[VEC];
             widen<DT, VEC>(pw[i], fw);
-            scale(s[i], rstd, fw, fy);
+#pragma unroll
+            for (int k = 0; k < VEC; ++k) fy[k] = s[i][k] * rstd * fw[k];
             store<UV, St::Stream>(yr + v * UV, narrow<DT, VEC>(fy));
         }
     }
