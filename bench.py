@@ -322,7 +322,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
                 "ms_per_step": round(e2e_ms / Ke, 3),
                 "how": f"pinned host -> device, kernels, device -> pinned host for every tensor of every step, in "
                        f"{chunk}-row chunks pipelined over three streams (upload / compute / download)"},
-        "gpu_launches": 6 * K,
+        "gpu_launches": 6 * K + 3 * Ke * (-(-T // chunk)),  # chain + per-kernel regions + chunked end-to-end steps
         "clocks": sampler.summary([(t_wall0, t_wall1), (t_wall2, t_wall3)]) if sampler else None,
     }
     if world == 1 and not args.no_sweep:

@@ -25,7 +25,7 @@ def test_bench_prints_one_json_line_with_the_contract_keys():
     assert r["n_gpus"] == 1 and r["steps"] == 5 and r["warmup"] == 3 and r["unit"] == "GB/s"
     assert r["higher_is_better"] is True and r["scaling"] == "weak" and r["vs_baseline"] is None
     assert r["dtype"] == "f32" and r["data"] == "synthetic" and "workload" in r["config"]
-    assert r["gpu_launches"] == 6 * 5 and r["value"] > 1000.0
+    assert r["gpu_launches"] == 6 * 5 + 3 * 2 * 4 and r["value"] > 1000.0  # + 2 end-to-end steps of 4 chunks
     rf = r["roofline"]
     assert rf["bound"] == "hbm" and rf["unit"] == "GB/s" and rf["peak"] > 0
     assert rf["frac"] == pytest.approx(rf["achieved"] / rf["peak"], rel=1e-3)
