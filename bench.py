@@ -160,7 +160,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
     torch.cuda.set_device(dev)
     from paper_2509_07506_b200 import build as astra_build
     if rank == 0:
-        astra_build.build()  # no-op when the library is newer than its sources; no fallback if it cannot be built
+        astra_build.ensure_built()  # no-op when the library is newer than its sources; a missing library is fatal
     if world > 1:
         dist.barrier()
     astra.load_library()  # fails loudly if the CUDA library is missing
@@ -333,7 +333,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
         result["fp32_variants"] = fp32_variants(astra, dev, peak)
     if world == 1 and not args.no_ablation:
         from paper_2509_07506_b200 import ablation
-        astra_build.build_ablation()
+        astra_build.ensure_built(ablation=True)
         abl = ablation.run("fp16", dev)
         result["ablation"] = {"what": "the paper's baseline/optimised design pairs (Section 5.3) rebuilt for sm_100a, "
                                       "timed beside this library on the Table 4 shapes and the three chain shapes",

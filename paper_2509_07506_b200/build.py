@@ -65,6 +65,20 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return _compile(LIB_PATH, SOURCES, force, verbose)
 
 
+def ensure_built(ablation: bool = False) -> str:
+    """Build if missing or stale; if the rebuild is impossible (no compiler on this machine) but a
+    built library is present, keep using it and say so.  A missing library is always an error."""
+    path = ABLATION_LIB_PATH if ablation else LIB_PATH
+    try:
+        return build_ablation() if ablation else build()
+    except Exception as exc:  # noqa: BLE001
+        if os.path.exists(path):
+            print(f"[astra build] could not rebuild {os.path.basename(path)} ({exc}); using the existing one",
+                  file=sys.stderr)
+            return path
+        raise
+
+
 def build_variant(lib_path: str, defines: dict) -> str:
     """Compile libastra's sources to `lib_path` with extra preprocessor definitions (used by the
     tests to lower the per-launch limits so that the multi-launch splitting runs on small inputs)."""

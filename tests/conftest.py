@@ -32,7 +32,7 @@ def _built_libraries():
     """Compile the CUDA libraries and the C oracle if they are missing or older than their sources
     (nvcc and gcc need no GPU), so that a fresh checkout can run either half of the suite."""
     from paper_2509_07506_b200 import build as astra_build
-    astra_build.build()
-    astra_build.build_ablation()
+    astra_build.ensure_built()
+    astra_build.ensure_built(ablation=True)
     import oracle
     oracle.build()
