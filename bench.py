@@ -600,7 +600,12 @@ def oracle_baseline(cfg, rows: int) -> dict:
     _oracle_pass(cfg, min(rows, 64), cores)  # load the library, touch the pages
     sec = min(_oracle_pass(cfg, rows, cores) for _ in range(2))
     b = sum(chain_bytes(rows).values())
-    return {"value": round(b / sec / 1e9, 3), "unit": UNIT, "cores": cores, "kind": "oracle",
+    # the same oracle on one core, on a smaller sample (it is ~cores times slower)
+    rows1 = max(1, min(rows, 512))
+    sec1 = _oracle_pass(cfg, rows1, 1)
+    single = {"value": round(sum(chain_bytes(rows1).values()) / sec1 / 1e9, 3), "unit": UNIT, "cores": 1,
+              "sample": f"first {rows1} rows/tokens, one pass, {sec1:.2f} s"}
+    return {"value": round(b / sec / 1e9, 3), "unit": UNIT, "cores": cores, "kind": "oracle", "single_thread": single,
             "sample": f"first {rows} rows/tokens of each of the three chain calls, best of 2 passes, "
                       f"{sec:.2f} s per pass, OpenMP over rows on all {cores} host cores",
             "seconds": round(sec, 3)}
