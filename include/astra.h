@@ -15,9 +15,18 @@
  *   - Pointers need only the natural alignment of their element (2 bytes for 16-bit values, 4 for
  *     fp32 values and for scores).  Wider alignment is detected and exploited inside; widths need not be multiples
  *     of 8.  A pointer with less than element alignment gives ASTRA_ERR_MISALIGNED.
- *   - Errors are return codes only: nothing is printed, thrown or aborted, and on any error
- *     nothing has been launched.  A zero-sized first dimension (T == 0) is ASTRA_OK and launches
- *     nothing; any other non-positive extent is ASTRA_ERR_BAD_SHAPE.
+ *   - Errors are return codes only: nothing is printed, thrown or aborted.  Arguments are checked
+ *     before anything is launched, so after any status other than ASTRA_OK and ASTRA_ERR_CUDA the
+ *     GPU has been given no work.  ASTRA_ERR_CUDA means the CUDA runtime refused a kernel launch
+ *     (the status is that launch's own return value).  Inputs beyond 2^31 - 1 vectors or rows are
+ *     issued as several launches; if one of them is refused the later ones are not issued, but
+ *     the earlier ones remain enqueued, so the outputs are then partly written.
+ *     The library links its own copy of the CUDA runtime: on success it neither reads nor clears
+ *     the runtime's per-thread "last error", and the caller's runtime state is never touched.
+ *   - A zero-sized first dimension (T == 0) is ASTRA_OK and launches nothing; the pointers of such
+ *     a call are not examined (an empty tensor may have a NULL address).  Any other non-positive
+ *     extent is ASTRA_ERR_BAD_SHAPE.  Limits: a fused_add_rmsnorm row holds at most 2^30 16-bit
+ *     units (2^30 bf16/fp16 or 2^29 fp32 elements); D of the other two operations is below 2^30.
  *   - Non-finite inputs never trap; they propagate by IEEE rules except where stated below.
  */
 #ifndef ASTRA_H_
@@ -151,6 +160,14 @@ astra_status_t astra_merge_attn_states_lse_ex(void *v_out, float *lse_out,
 
 /* Static, NUL-terminated description of a status code (never NULL). */
 const char *astra_status_string(astra_status_t status);
+
+/*
+ * Static, NUL-terminated identifier of the sources this library was compiled from: the hexadecimal
+ * SHA-256 the build script computes over the headers and CUDA sources ("unidentified" if the
+ * library was compiled by hand).  The Python binding compares it with the sources beside it when it
+ * loads the library and refuses a library built from other sources.  No counterpart in the paper.
+ */
+const char *astra_build_id(void);
 
 #ifdef __cplusplus
 }

@@ -12,7 +12,9 @@ results as ``float64`` (and ``uint16`` for the bit-exact residual).
 from __future__ import annotations
 
 import ctypes
+import hashlib
 import os
+import re
 import subprocess
 
 import numpy as np
@@ -27,18 +29,34 @@ _LIB = os.path.join(_HERE, "liboracle.so")
 _lib = None
 
 
+def _source_hash(src: str) -> str:
+    with open(src, "rb") as fh:
+        return hashlib.sha256(fh.read()).hexdigest()
+
+
 def compile_source(src: str, out: str) -> str:
-    """gcc command used for the oracle (no fast-math, no contraction)."""
+    """gcc command used for the oracle (no fast-math, no contraction).  The hash of the source is
+    compiled in, so that a built library can be matched to the source beside it by content."""
     subprocess.check_call(
         ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared",
-         "-ffp-contract=off", "-fno-fast-math", "-o", out, src, "-lm"]
+         "-ffp-contract=off", "-fno-fast-math", f'-DORACLE_BUILD_ID="{_source_hash(src)}"', "-o", out, src, "-lm"]
     )
     return out
 
 
+def _embedded_hash(lib: str):
+    try:
+        with open(lib, "rb") as fh:
+            m = re.search(rb"oracle-build-id:([0-9a-f]{64})", fh.read())
+    except OSError:
+        return None
+    return m.group(1).decode() if m else None
+
+
 def build(force: bool = False) -> str:
-    """Compile the oracle with gcc; returns the path of the shared object."""
-    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    """Compile the oracle with gcc unless the built library already matches the source; returns the
+    path of the shared object."""
+    stale = _embedded_hash(_LIB) != _source_hash(_SRC)
     if force or stale:
         tmp = _LIB + f".tmp{os.getpid()}"
         compile_source(_SRC, tmp)

@@ -31,6 +31,12 @@
 #include <stdint.h>
 #include <string.h>
 
+#ifndef ORACLE_BUILD_ID
+#define ORACLE_BUILD_ID "unidentified"
+#endif
+/* hash of this file as compiled (set by the build script), findable in the built library */
+const char oracle_build_marker[] = "oracle-build-id:" ORACLE_BUILD_ID;
+
 #define ORACLE_BF16 0
 #define ORACLE_FP16 1
 #define ORACLE_FP32 2 /* IEEE binary32 storage: patterns are 32 bits wide */

@@ -36,6 +36,7 @@ EXPORTED_SYMBOLS = (
     "astra_silu_and_mul_ex",
     "astra_merge_attn_states_lse_ex",
     "astra_status_string",
+    "astra_build_id",
 )
 
 _DTYPE_CODE = {torch.bfloat16: ASTRA_BF16, torch.float16: ASTRA_FP16, torch.float32: ASTRA_FP32}
@@ -76,17 +77,41 @@ def load_library() -> ctypes.CDLL:
     lib.astra_merge_attn_states_lse_ex.restype = i32
     lib.astra_status_string.argtypes = [i32]
     lib.astra_status_string.restype = ctypes.c_char_p
+    lib.astra_build_id.argtypes = []
+    lib.astra_build_id.restype = ctypes.c_char_p
+    _refuse_stale(lib)
     _lib = lib
     return lib
+
+
+def _refuse_stale(lib) -> None:
+    """Where the library sits beside its sources (a source checkout), it must have been built from
+    exactly those sources: the hash compiled into it is compared with the hash of the files."""
+    from . import build as _build
+    if not (os.path.isdir(_build.CSRC) and os.path.isdir(_build.INCLUDE)):
+        return
+    built_from, on_disk = lib.astra_build_id().decode(), _build.source_hash()
+    if built_from != on_disk:
+        raise ImportError(
+            f"{LIB_PATH} was built from other sources (library {built_from[:12]}, sources {on_disk[:12]}): "
+            "rebuild it with `python -m paper_2509_07506_b200.build`")
 
 
 def status_string(status: int) -> str:
     return load_library().astra_status_string(int(status)).decode()
 
 
-def _check(t: torch.Tensor, name: str, dtype=None, shape=None) -> None:
+def _same_device(t: torch.Tensor, name: str, device) -> None:
+    """Every operand of a call must live on one GPU: the C side receives bare addresses and launches on
+    that GPU, so a tensor from another one would be dereferenced as a foreign (or unmapped) address."""
+    if device is not None and t.device != device:
+        raise ValueError(f"{name} is on {t.device}, but the call's first tensor is on {device}")
+
+
+def _check(t: torch.Tensor, name: str, dtype=None, shape=None, device=None) -> None:
     if not isinstance(t, torch.Tensor) or not t.is_cuda:
         raise TypeError(f"{name} must be a CUDA tensor")
+    _same_device(t, name, device)
     if not t.is_contiguous():
         raise ValueError(f"{name} must be contiguous")
     if dtype is not None and t.dtype != dtype:
@@ -136,38 +161,110 @@ class _on_device:
         return False
 
 
-def astra_fused_add_rmsnorm(x: torch.Tensor, residual: torch.Tensor, weight: torch.Tensor,
-                            eps: float, stream: Optional[torch.cuda.Stream] = None) -> None:
-    """In place: residual <- x + residual, x <- RMSNorm(x + residual) * weight.  x, residual [T, H]."""
+class PreparedCall:
+    """One validated call, kept ready to be issued again.
+
+    The plain functions below check every tensor, read its address and convert the arguments on
+    each call; for the small shapes of decode steps that host work takes longer than the kernel.
+    A prepared call does all of it once: it keeps the library function and the converted argument
+    tuple (and references to the tensors, so their addresses stay valid) and ``__call__`` only looks
+    up the current stream and issues the launch.  The tensors' contents may change between calls;
+    their addresses, shapes and dtypes are fixed at preparation.  Results are identical to the plain
+    call's, which is itself ``prepare(...)()``.
+    """
+
+    __slots__ = ("name", "_fn", "_args", "_device", "_keep")
+
+    def __init__(self, name: str, fn, args: tuple, device: torch.device, keep: tuple):
+        self.name = name
+        self._fn = fn
+        self._args = args
+        self._device = device.index if device.index is not None else torch.cuda.current_device()
+        self._keep = keep
+
+    def __call__(self, stream: Optional[torch.cuda.Stream] = None) -> None:
+        dev = self._device
+        if stream is not None:
+            handle = stream.cuda_stream
+        elif _raw_current_stream is not None:
+            handle = _raw_current_stream(dev)
+        else:
+            handle = torch.cuda.current_stream(dev).cuda_stream
+        if _raw_current_device() == dev:
+            st = self._fn(*self._args, handle)
+        else:  # the C side launches on the current device
+            with torch.cuda.device(dev):
+                st = self._fn(*self._args, handle)
+        if st != ASTRA_OK:
+            raise AstraError(st, self.name)
+
+
+_raw_current_device = getattr(torch._C, "_cuda_getDevice", None) or torch.cuda.current_device
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def prepare_fused_add_rmsnorm(x: torch.Tensor, residual: torch.Tensor, weight: torch.Tensor,
+                              eps: float) -> PreparedCall:
+    """Validated, re-issuable form of :func:`astra_fused_add_rmsnorm`."""
     _check(x, "x")
     code = _code(x, "x")
     if x.dim() != 2:
         raise ValueError("x must be [T, H]")
     T, H = x.shape
-    _check(residual, "residual", x.dtype, (T, H))
-    _check(weight, "weight", x.dtype, (H,))
-    with _on_device(x):
-        st = load_library().astra_fused_add_rmsnorm(
-            x.data_ptr(), residual.data_ptr(), weight.data_ptr(), T, H, float(eps), code,
-            _stream(x, stream))
-    if st != ASTRA_OK:
-        raise AstraError(st, "astra_fused_add_rmsnorm")
+    _check(residual, "residual", x.dtype, (T, H), x.device)
+    _check(weight, "weight", x.dtype, (H,), x.device)
+    args = (_ptr(x), _ptr(residual), _ptr(weight), ctypes.c_int64(T), ctypes.c_int64(H),
+            ctypes.c_float(float(eps)), ctypes.c_int(code))
+    return PreparedCall("astra_fused_add_rmsnorm", load_library().astra_fused_add_rmsnorm, args, x.device,
+                        (x, residual, weight))
 
 
-def astra_silu_and_mul(out: torch.Tensor, input: torch.Tensor,
-                       stream: Optional[torch.cuda.Stream] = None) -> None:
-    """out[T, D] <- SiLU(input[:, :D]) * input[:, D:]."""
+def astra_fused_add_rmsnorm(x: torch.Tensor, residual: torch.Tensor, weight: torch.Tensor,
+                            eps: float, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """In place: residual <- x + residual, x <- RMSNorm(x + residual) * weight.  x, residual [T, H]."""
+    prepare_fused_add_rmsnorm(x, residual, weight, eps)(stream)
+
+
+def prepare_silu_and_mul(out: torch.Tensor, input: torch.Tensor) -> PreparedCall:
+    """Validated, re-issuable form of :func:`astra_silu_and_mul`."""
     _check(input, "input")
     code = _code(input, "input")
     if input.dim() != 2 or input.shape[1] % 2:
         raise ValueError("input must be [T, 2*D]")
     T, D = input.shape[0], input.shape[1] // 2
-    _check(out, "out", input.dtype, (T, D))
-    with _on_device(input):
-        st = load_library().astra_silu_and_mul(out.data_ptr(), input.data_ptr(), T, D, code,
-                                               _stream(input, stream))
-    if st != ASTRA_OK:
-        raise AstraError(st, "astra_silu_and_mul")
+    _check(out, "out", input.dtype, (T, D), input.device)
+    args = (_ptr(out), _ptr(input), ctypes.c_int64(T), ctypes.c_int64(D), ctypes.c_int(code))
+    return PreparedCall("astra_silu_and_mul", load_library().astra_silu_and_mul, args, input.device, (out, input))
+
+
+def astra_silu_and_mul(out: torch.Tensor, input: torch.Tensor,
+                       stream: Optional[torch.cuda.Stream] = None) -> None:
+    """out[T, D] <- SiLU(input[:, :D]) * input[:, D:]."""
+    prepare_silu_and_mul(out, input)(stream)
+
+
+def prepare_merge_attn_states_lse(v_out: torch.Tensor, lse_out: Optional[torch.Tensor],
+                                  v_a: torch.Tensor, lse_a: torch.Tensor,
+                                  v_b: torch.Tensor, lse_b: torch.Tensor) -> PreparedCall:
+    """Validated, re-issuable form of :func:`astra_merge_attn_states_lse`."""
+    _check(v_a, "v_a")
+    code = _code(v_a, "v_a")
+    if v_a.dim() != 3:
+        raise ValueError("v_a must be [T, Hh, D]")
+    T, Hh, D = v_a.shape
+    _check(v_b, "v_b", v_a.dtype, (T, Hh, D), v_a.device)
+    _check(v_out, "v_out", v_a.dtype, (T, Hh, D), v_a.device)
+    _check(lse_a, "lse_a", torch.float32, (T, Hh), v_a.device)
+    _check(lse_b, "lse_b", torch.float32, (T, Hh), v_a.device)
+    if lse_out is not None:
+        _check(lse_out, "lse_out", torch.float32, (T, Hh), v_a.device)
+    args = (_ptr(v_out), _ptr(lse_out), _ptr(v_a), _ptr(lse_a), _ptr(v_b), _ptr(lse_b),
+            ctypes.c_int64(T), ctypes.c_int64(Hh), ctypes.c_int64(D), ctypes.c_int(code))
+    return PreparedCall("astra_merge_attn_states_lse", load_library().astra_merge_attn_states_lse, args,
+                        v_a.device, (v_out, lse_out, v_a, lse_a, v_b, lse_b))
 
 
 def astra_merge_attn_states_lse(v_out: torch.Tensor, lse_out: Optional[torch.Tensor],
@@ -175,32 +272,16 @@ def astra_merge_attn_states_lse(v_out: torch.Tensor, lse_out: Optional[torch.Ten
                                 v_b: torch.Tensor, lse_b: torch.Tensor,
                                 stream: Optional[torch.cuda.Stream] = None) -> None:
     """v_out, lse_out <- merge of (v_a, lse_a) and (v_b, lse_b).  v_* [T, Hh, D]; lse_* [T, Hh] fp32."""
-    _check(v_a, "v_a")
-    code = _code(v_a, "v_a")
-    if v_a.dim() != 3:
-        raise ValueError("v_a must be [T, Hh, D]")
-    T, Hh, D = v_a.shape
-    _check(v_b, "v_b", v_a.dtype, (T, Hh, D))
-    _check(v_out, "v_out", v_a.dtype, (T, Hh, D))
-    _check(lse_a, "lse_a", torch.float32, (T, Hh))
-    _check(lse_b, "lse_b", torch.float32, (T, Hh))
-    if lse_out is not None:
-        _check(lse_out, "lse_out", torch.float32, (T, Hh))
-    with _on_device(v_a):
-        st = load_library().astra_merge_attn_states_lse(
-            v_out.data_ptr(), lse_out.data_ptr() if lse_out is not None else None,
-            v_a.data_ptr(), lse_a.data_ptr(), v_b.data_ptr(), lse_b.data_ptr(),
-            T, Hh, D, code, _stream(v_a, stream))
-    if st != ASTRA_OK:
-        raise AstraError(st, "astra_merge_attn_states_lse")
+    prepare_merge_attn_states_lse(v_out, lse_out, v_a, lse_a, v_b, lse_b)(stream)
 
 
 # ---- strided / out-of-place forms ---------------------------------------------------------------
 
-def _check_rows(t: torch.Tensor, name: str, dtype, shape) -> None:
+def _check_rows(t: torch.Tensor, name: str, dtype, shape, device=None) -> None:
     """A tensor whose innermost dimension is contiguous; outer strides are free (non-negative)."""
     if not isinstance(t, torch.Tensor) or not t.is_cuda:
         raise TypeError(f"{name} must be a CUDA tensor")
+    _same_device(t, name, device)
     if dtype is not None and t.dtype != dtype:
         raise TypeError(f"{name} must have dtype {dtype}, got {t.dtype}")
     if tuple(t.shape) != tuple(shape):
@@ -226,8 +307,8 @@ def astra_fused_add_rmsnorm_ex(y: torch.Tensor, residual_out: torch.Tensor, x: t
     code = _code(x, "x")
     T, H = x.shape
     for t, n in ((x, "x"), (residual, "residual"), (y, "y"), (residual_out, "residual_out")):
-        _check_rows(t, n, x.dtype, (T, H))
-    _check(weight, "weight", x.dtype, (H,))
+        _check_rows(t, n, x.dtype, (T, H), x.device)
+    _check(weight, "weight", x.dtype, (H,), x.device)
     with _on_device(x):
         st = load_library().astra_fused_add_rmsnorm_ex(
             y.data_ptr(), residual_out.data_ptr(), x.data_ptr(), residual.data_ptr(), weight.data_ptr(),
@@ -245,7 +326,7 @@ def astra_silu_and_mul_ex(out: torch.Tensor, gate: torch.Tensor, up: torch.Tenso
     code = _code(gate, "gate")
     T, D = gate.shape
     for t, n in ((gate, "gate"), (up, "up"), (out, "out")):
-        _check_rows(t, n, gate.dtype, (T, D))
+        _check_rows(t, n, gate.dtype, (T, D), gate.device)
     with _on_device(gate):
         st = load_library().astra_silu_and_mul_ex(out.data_ptr(), gate.data_ptr(), up.data_ptr(), T, D,
                                                   _pitch(out), _pitch(gate), _pitch(up), code,
@@ -265,11 +346,12 @@ def astra_merge_attn_states_lse_ex(v_out: torch.Tensor, lse_out: Optional[torch.
     code = _code(v_a, "v_a")
     T, Hh, D = v_a.shape
     for t, n in ((v_a, "v_a"), (v_b, "v_b"), (v_out, "v_out")):
-        _check_rows(t, n, v_a.dtype, (T, Hh, D))
+        _check_rows(t, n, v_a.dtype, (T, Hh, D), v_a.device)
     scores = [(lse_a, "lse_a"), (lse_b, "lse_b")] + ([(lse_out, "lse_out")] if lse_out is not None else [])
     for t, n in scores:
         if not isinstance(t, torch.Tensor) or not t.is_cuda or t.dtype != torch.float32:
             raise TypeError(f"{n} must be a float32 CUDA tensor")
+        _same_device(t, n, v_a.device)
         if tuple(t.shape) != (T, Hh) or any(s < 0 for s in t.stride()):
             raise ValueError(f"{n} must have shape {(T, Hh)} and non-negative strides")
     so = (lse_out.stride(0), lse_out.stride(1)) if lse_out is not None else (0, 0)

@@ -5,7 +5,9 @@ to this file; nothing is installed outside the source tree.
 """
 from __future__ import annotations
 
+import hashlib
 import os
+import re
 import shutil
 import subprocess
 import sys
@@ -40,18 +42,46 @@ def _inputs():
     return files
 
 
-def is_stale(lib_path: str = LIB_PATH) -> bool:
-    if not os.path.exists(lib_path):
-        return True
-    built = os.path.getmtime(lib_path)
-    return any(os.path.getmtime(f) > built for f in _inputs())
+_ID_MARKER = b"astra-build-id:"
+
+
+def source_hash(extra_flags=()) -> str:
+    """SHA-256 over the names and contents of every header and CUDA source (and the extra compiler
+    flags of a variant build).  It is compiled into each library, so a library can be matched to the
+    sources beside it by content; file times, which a copy or a checkout rewrites, play no part."""
+    h = hashlib.sha256()
+    for path in sorted(_inputs()):
+        h.update(os.path.basename(path).encode() + b"\0")
+        with open(path, "rb") as fh:
+            h.update(fh.read())
+        h.update(b"\0")
+    for flag in extra_flags:
+        h.update(flag.encode() + b"\0")
+    return h.hexdigest()
+
+
+def embedded_hash(lib_path: str):
+    """The source hash compiled into a built library (read from the file, without loading it), or None."""
+    try:
+        with open(lib_path, "rb") as fh:
+            blob = fh.read()
+    except OSError:
+        return None
+    m = re.search(re.escape(_ID_MARKER) + rb"([0-9a-f]{64})", blob)
+    return m.group(1).decode() if m else None
+
+
+def is_stale(lib_path: str = LIB_PATH, extra_flags=()) -> bool:
+    """True when the library is missing or was not built from the sources now on disk."""
+    return embedded_hash(lib_path) != source_hash(extra_flags)
 
 
 def _compile(lib_path: str, sources, force: bool, verbose: bool, extra_flags=()) -> str:
-    if not force and not is_stale(lib_path):
+    if not force and not is_stale(lib_path, extra_flags):
         return lib_path
     tmp = lib_path + f".tmp{os.getpid()}"
-    cmd = [_nvcc(), *NVCC_FLAGS, *extra_flags, "-I", INCLUDE, "-I", CSRC, "-o", tmp]
+    cmd = [_nvcc(), *NVCC_FLAGS, *extra_flags, f'-DASTRA_BUILD_ID="{source_hash(extra_flags)}"',
+           "-I", INCLUDE, "-I", CSRC, "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in sources]
@@ -61,29 +91,22 @@ def _compile(lib_path: str, sources, force: bool, verbose: bool, extra_flags=())
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile libastra.so if it is missing or older than any source; returns its path."""
+    """Compile libastra.so if it is missing or was built from other sources; returns its path."""
     return _compile(LIB_PATH, SOURCES, force, verbose)
 
 
 def ensure_built(ablation: bool = False) -> str:
-    """Build if missing or stale; if the rebuild is impossible (no compiler on this machine) but a
-    built library is present, keep using it and say so.  A missing library is always an error."""
-    path = ABLATION_LIB_PATH if ablation else LIB_PATH
-    try:
-        return build_ablation() if ablation else build()
-    except Exception as exc:  # noqa: BLE001
-        if os.path.exists(path):
-            print(f"[astra build] could not rebuild {os.path.basename(path)} ({exc}); using the existing one",
-                  file=sys.stderr)
-            return path
-        raise
+    """Build if the library is missing or does not match the sources on disk.  A library that cannot
+    be rebuilt (no compiler on this machine) and does not match is an error: results must never come
+    from a library other than the one the sources describe."""
+    return build_ablation() if ablation else build()
 
 
 def build_variant(lib_path: str, defines: dict) -> str:
     """Compile libastra's sources to `lib_path` with extra preprocessor definitions (used by the
     tests to lower the per-launch limits so that the multi-launch splitting runs on small inputs)."""
-    flags = [f"-D{k}={v}" for k, v in defines.items()]
-    return _compile(lib_path, SOURCES, True, False, flags)
+    flags = [f"-D{k}={v}" for k, v in sorted(defines.items())]
+    return _compile(lib_path, SOURCES, False, False, flags)
 
 
 def build_ablation(force: bool = False, verbose: bool = False) -> str:

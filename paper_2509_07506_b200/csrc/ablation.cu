@@ -1,186 +1,249 @@
-// Ablation library (declared in astra_ablation.h): the baseline / optimised design pairs described
-// in the paper's case studies (Section 5.3, Figures 2-5), written from those descriptions for
-// sm_100a.  They exist to be timed against each other and against the library's own kernels; they
-// use the same arithmetic readings (binary32 throughout, one rounding per store) so the same parity
-// gates apply.
+// Ablation library (declared in astra_ablation.h).  The paper's case studies (Section 5.3) explain
+// its speedups by three contrasts: loop-invariant weights recomputed per element vs derived once;
+// a block reduction done entirely in shared memory vs in registers with a short shared-memory
+// finish; scalar 16-bit accesses with library math vs 32-bit accesses with fast-math intrinsics.
+// Each contrast is built here as a pair of kernels that differ in that one respect only, so the
+// effect can be timed on sm_100a.  The kernels are this library's own (grid-stride work
+// distribution, block size as a template parameter, reductions that accept any block size); they
+// follow the arithmetic readings of the main library (binary32 throughout, one rounding per store)
+// so the same parity gates apply.
 #include <cuda_runtime.h>
 
 #include "astra_ablation.h"
 #include "vec.cuh"
 
+#ifndef ASTRA_BUILD_ID
+#define ASTRA_BUILD_ID "unidentified"
+#endif
+// hash of the sources this library was compiled from; the build script finds it in the file
+extern "C" __attribute__((used, visibility("default"))) const char astra_ablation_build_marker[] =
+    "astra-build-id:" ASTRA_BUILD_ID;
+
 namespace {
 
 using namespace astra;
 
-constexpr int kThreads = 256;
+constexpr int kBlock = 256;        // threads per block of every kernel here
+constexpr int kWavesOfBlocks = 8;  // grid-stride kernels launch at most this many blocks per SM
 
 // ---------------------------------------------------------------------------------------------
-// Kernel 1: merge_attn_states_lse.  One warp per (token, head) row; lanes stride over head_dim.
+// Kernel 1: merge_attn_states_lse.  A warp walks over (token, head) rows; its lanes cover head_dim.
 // ---------------------------------------------------------------------------------------------
-struct Weights { float a, b, lse; };
+struct Mix {
+    float a, b;  // softmax of the two scores
+    float lse;   // log(e^{Sa} + e^{Sb})
+};
 
-// max, two exponentials, one division: the weight computation the paper's Figure 2 hoists.
-__device__ __forceinline__ Weights mixing_weights(float sa, float sb) {
-    Weights w;
-    const float m = fmaxf(sa, sb);
-    if (m == -INFINITY) { w.a = 0.f; w.b = 0.f; w.lse = -INFINITY; return w; }
-    const float ea = expf(sa - m), eb = expf(sb - m);
-    const float inv = 1.0f / (ea + eb);
-    w.a = ea * inv;
-    w.b = eb * inv;
-    w.lse = m + logf(ea + eb);
-    return w;
+// Two-way softmax shifted by the larger score (nothing overflows), with library exponentials and
+// true divisions: this is the per-row work whose placement the two designs differ in.
+__device__ __forceinline__ Mix mix_of(float sa, float sb) {
+    const float top = fmaxf(sa, sb);
+    if (top == -INFINITY) return Mix{0.f, 0.f, -INFINITY};  // both states empty
+    const float ea = expf(sa - top), eb = expf(sb - top);
+    const float z = ea + eb;
+    return Mix{ea / z, eb / z, top + logf(z)};
 }
 
-__device__ __forceinline__ float blend(const Weights &w, float va, float vb) {
-    // a zero weight drops its side (an empty state may hold anything)
-    const float ta = (w.a == 0.f) ? 0.f : w.a * va;
-    return (w.b == 0.f) ? ta : fmaf(w.b, vb, ta);
-}
-
-// design 0: the weights are recomputed for every element inside the loop over head_dim
-template <int DT>
-__global__ void __launch_bounds__(kThreads)
-merge_recompute_kernel(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
-                       const uint16_t *v_b, const float *lse_b, int64_t rows, int D) {
-    const int64_t row = static_cast<int64_t>(blockIdx.x) * (kThreads / 32) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (row >= rows) return;
-    const float sa = lse_a[row], sb = lse_b[row];
-    const uint16_t *pa = v_a + row * D, *pb = v_b + row * D;
-    uint16_t *po = v_out + row * D;
-    for (int d = lane; d < D; d += 32) {
-        const Weights w = mixing_weights(sa, sb);  // loop-invariant, recomputed on purpose
-        po[d] = Storage<DT>::narrow1(blend(w, Storage<DT>::widen1(pa[d]), Storage<DT>::widen1(pb[d])));
-        if (d == 0) lse_out[row] = w.lse;
-    }
-}
-
-// design 1: weights once per row, then a light loop; two elements per 32-bit access
-template <int DT>
-__global__ void __launch_bounds__(kThreads)
-merge_hoisted_kernel(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
-                     const uint16_t *v_b, const float *lse_b, int64_t rows, int D) {
-    const int64_t row = static_cast<int64_t>(blockIdx.x) * (kThreads / 32) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (row >= rows) return;
-    const Weights w = mixing_weights(lse_a[row], lse_b[row]);
-    const uint32_t *pa = reinterpret_cast<const uint32_t *>(v_a + row * D);
-    const uint32_t *pb = reinterpret_cast<const uint32_t *>(v_b + row * D);
-    uint32_t *po = reinterpret_cast<uint32_t *>(v_out + row * D);
-    for (int d = lane; d < D / 2; d += 32) {
-        float a0, a1, b0, b1;
-        Storage<DT>::widen2(pa[d], a0, a1);
-        Storage<DT>::widen2(pb[d], b0, b1);
-        po[d] = Storage<DT>::narrow2(blend(w, a0, b0), blend(w, a1, b1));
-    }
-    if (lane == 0) lse_out[row] = w.lse;
-}
-
-// ---------------------------------------------------------------------------------------------
-// Kernel 2: fused_add_rmsnorm, one block per row, two sweeps over the row (the sum of squares
-// first, then the outputs; nothing is written before the norm is known).
-// ---------------------------------------------------------------------------------------------
-
-// design 0: tree reduction in shared memory, one block barrier per halving step
-template <int DT>
-__global__ void __launch_bounds__(kThreads)
-rmsnorm_tree_kernel(uint16_t *x, uint16_t *residual, const uint16_t *weight, int H, float eps) {
-    __shared__ float partial[kThreads];
-    uint16_t *xr = x + static_cast<int64_t>(blockIdx.x) * H;
-    uint16_t *rr = residual + static_cast<int64_t>(blockIdx.x) * H;
-    const int tx = threadIdx.x;
+// A side of weight zero is left out altogether: an empty state may hold anything.
+__device__ __forceinline__ float blend(const Mix &m, float va, float vb) {
     float acc = 0.f;
-    for (int j = tx; j < H; j += kThreads) {
-        const float s = Storage<DT>::widen1(xr[j]) + Storage<DT>::widen1(rr[j]);
-        acc = fmaf(s, s, acc);
+    if (m.a != 0.f) acc = m.a * va;
+    if (m.b != 0.f) acc = fmaf(m.b, vb, acc);
+    return acc;
+}
+
+// HOIST = false: the scores are fetched and the weights derived again for every element (the stores
+// in between may alias the scores, so the compiler cannot lift them out either); 16-bit accesses.
+// HOIST = true: once per row, ahead of the element loop, which then moves two elements per access.
+template <int DT, bool HOIST, int BLOCK>
+__global__ void __launch_bounds__(BLOCK)
+merge_pair_kernel(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
+                  const uint16_t *v_b, const float *lse_b, int64_t rows, int D) {
+    constexpr int kWarps = BLOCK / 32;
+    const int lane = threadIdx.x % 32;
+    const int64_t first = static_cast<int64_t>(blockIdx.x) * kWarps + threadIdx.x / 32;
+    const int64_t step = static_cast<int64_t>(gridDim.x) * kWarps;
+    for (int64_t row = first; row < rows; row += step) {
+        const int64_t at = row * D;
+        if constexpr (HOIST) {
+            const Mix m = mix_of(lse_a[row], lse_b[row]);
+            const uint32_t *pa = reinterpret_cast<const uint32_t *>(v_a + at);
+            const uint32_t *pb = reinterpret_cast<const uint32_t *>(v_b + at);
+            uint32_t *po = reinterpret_cast<uint32_t *>(v_out + at);
+            for (int p = lane; 2 * p < D; p += 32) {
+                float a_lo, a_hi, b_lo, b_hi;
+                Storage<DT>::widen2(pa[p], a_lo, a_hi);
+                Storage<DT>::widen2(pb[p], b_lo, b_hi);
+                po[p] = Storage<DT>::narrow2(blend(m, a_lo, b_lo), blend(m, a_hi, b_hi));
+            }
+            if (lane == 0) lse_out[row] = m.lse;
+        } else {
+            for (int d = lane; d < D; d += 32) {
+                const Mix m = mix_of(lse_a[row], lse_b[row]);
+                v_out[at + d] = Storage<DT>::narrow1(
+                    blend(m, Storage<DT>::widen1(v_a[at + d]), Storage<DT>::widen1(v_b[at + d])));
+                if (d == 0) lse_out[row] = m.lse;
+            }
+        }
     }
-    partial[tx] = acc;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Kernel 2: fused_add_rmsnorm.  A block walks over rows; each row is swept twice (sum of squares,
+// then the outputs, so nothing is written before the norm is known).  The pair differs in how the
+// per-thread partial sums become the row total, and in the access width.
+// ---------------------------------------------------------------------------------------------
+
+// All-shared-memory reduction: every partial goes to shared memory and the live range is folded
+// onto its lower part, with a block barrier after each fold, until one value is left.  Any BLOCK
+// (an odd live range keeps its middle element for the next fold).
+template <int BLOCK>
+__device__ __forceinline__ float total_in_shared_memory(float mine, float *scratch) {
+    scratch[threadIdx.x] = mine;
     __syncthreads();
-    for (int half = kThreads / 2; half > 0; half >>= 1) {
-        if (tx < half) partial[tx] += partial[tx + half];
+    int live = BLOCK;
+    while (live > 1) {
+        const int kept = (live + 1) / 2;
+        if (static_cast<int>(threadIdx.x) + kept < live) scratch[threadIdx.x] += scratch[threadIdx.x + kept];
         __syncthreads();
+        live = kept;
     }
-    const float rstd = rsqrtf(partial[0] / static_cast<float>(H) + eps);
-    for (int j = tx; j < H; j += kThreads) {
-        const float s = Storage<DT>::widen1(xr[j]) + Storage<DT>::widen1(rr[j]);
-        rr[j] = Storage<DT>::narrow1(s);
-        xr[j] = Storage<DT>::narrow1(s * rstd * Storage<DT>::widen1(weight[j]));
-    }
+    const float total = scratch[0];
+    __syncthreads();  // scratch is reused by the next row
+    return total;
 }
 
-// design 1: shuffles inside each warp, one shared slot per warp, short finish; 32-bit accesses
-template <int DT>
-__global__ void __launch_bounds__(kThreads)
-rmsnorm_shuffle_kernel(uint16_t *x, uint16_t *residual, const uint16_t *weight, int H, float eps) {
-    __shared__ float warp_sum[kThreads / 32];
-    uint32_t *xr = reinterpret_cast<uint32_t *>(x + static_cast<int64_t>(blockIdx.x) * H);
-    uint32_t *rr = reinterpret_cast<uint32_t *>(residual + static_cast<int64_t>(blockIdx.x) * H);
-    const uint32_t *wr = reinterpret_cast<const uint32_t *>(weight);
-    const int tx = threadIdx.x, lane = tx & 31, warp = tx >> 5;
-    float acc = 0.f;
-    for (int j = tx; j < H / 2; j += kThreads) {
-        float x0, x1, r0, r1;
-        Storage<DT>::widen2(xr[j], x0, x1);
-        Storage<DT>::widen2(rr[j], r0, r1);
-        const float s0 = x0 + r0, s1 = x1 + r1;
-        acc = fmaf(s0, s0, acc);
-        acc = fmaf(s1, s1, acc);
-    }
-    for (int off = 16; off > 0; off >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, off);
-    if (lane == 0) warp_sum[warp] = acc;
+// Register reduction: a butterfly of shuffles leaves the warp's sum in every lane; one value per
+// warp passes through shared memory, and the first warp's butterfly over those finishes the job.
+template <int BLOCK>
+__device__ __forceinline__ float total_in_registers(float mine, float *per_warp) {
+    static_assert(BLOCK % 32 == 0 && BLOCK <= 1024, "whole warps, at most 32 of them");
+    constexpr int kWarps = BLOCK / 32;
+    for (int mask = 1; mask < 32; mask <<= 1) mine += __shfl_xor_sync(0xffffffffu, mine, mask);
+    if (threadIdx.x % 32 == 0) per_warp[threadIdx.x / 32] = mine;
     __syncthreads();
-    float total = 0.f;
-#pragma unroll
-    for (int i = 0; i < kThreads / 32; ++i) total += warp_sum[i];
-    const float rstd = rsqrtf(total / static_cast<float>(H) + eps);
-    for (int j = tx; j < H / 2; j += kThreads) {
-        float x0, x1, r0, r1, w0, w1;
-        Storage<DT>::widen2(xr[j], x0, x1);
-        Storage<DT>::widen2(rr[j], r0, r1);
-        Storage<DT>::widen2(wr[j], w0, w1);
-        const float s0 = x0 + r0, s1 = x1 + r1;
-        rr[j] = Storage<DT>::narrow2(s0, s1);
-        xr[j] = Storage<DT>::narrow2(s0 * rstd * w0, s1 * rstd * w1);
+    float t = (threadIdx.x % 32) < kWarps ? per_warp[threadIdx.x % 32] : 0.f;
+    for (int mask = 1; mask < 32; mask <<= 1) t += __shfl_xor_sync(0xffffffffu, t, mask);
+    __syncthreads();  // per_warp is reused by the next row
+    return t;
+}
+
+template <int DT, bool REGISTERS, int BLOCK>
+__global__ void __launch_bounds__(BLOCK)
+rmsnorm_pair_kernel(uint16_t *x, uint16_t *residual, const uint16_t *weight, int64_t T, int H, float eps) {
+    __shared__ float scratch[REGISTERS ? 32 : BLOCK];
+    const float inv_H = 1.0f / static_cast<float>(H);
+    for (int64_t row = blockIdx.x; row < T; row += gridDim.x) {
+        uint16_t *xr = x + row * H, *rr = residual + row * H;
+        float sq = 0.f;
+        float rstd;
+        if constexpr (REGISTERS) {
+            uint32_t *x2 = reinterpret_cast<uint32_t *>(xr), *r2 = reinterpret_cast<uint32_t *>(rr);
+            const uint32_t *w2 = reinterpret_cast<const uint32_t *>(weight);
+            for (int p = threadIdx.x; 2 * p < H; p += BLOCK) {
+                float xa, xb, ra, rb;
+                Storage<DT>::widen2(x2[p], xa, xb);
+                Storage<DT>::widen2(r2[p], ra, rb);
+                const float sa = xa + ra, sb = xb + rb;
+                sq = fmaf(sa, sa, sq);
+                sq = fmaf(sb, sb, sq);
+            }
+            rstd = rsqrtf(fmaf(total_in_registers<BLOCK>(sq, scratch), inv_H, eps));
+            for (int p = threadIdx.x; 2 * p < H; p += BLOCK) {
+                float xa, xb, ra, rb, wa, wb;
+                Storage<DT>::widen2(x2[p], xa, xb);
+                Storage<DT>::widen2(r2[p], ra, rb);
+                Storage<DT>::widen2(w2[p], wa, wb);
+                const float sa = xa + ra, sb = xb + rb;
+                r2[p] = Storage<DT>::narrow2(sa, sb);
+                x2[p] = Storage<DT>::narrow2(sa * rstd * wa, sb * rstd * wb);
+            }
+        } else {
+            for (int j = threadIdx.x; j < H; j += BLOCK) {
+                const float s = Storage<DT>::widen1(xr[j]) + Storage<DT>::widen1(rr[j]);
+                sq = fmaf(s, s, sq);
+            }
+            rstd = rsqrtf(fmaf(total_in_shared_memory<BLOCK>(sq, scratch), inv_H, eps));
+            for (int j = threadIdx.x; j < H; j += BLOCK) {
+                const float s = Storage<DT>::widen1(xr[j]) + Storage<DT>::widen1(rr[j]);
+                rr[j] = Storage<DT>::narrow1(s);
+                xr[j] = Storage<DT>::narrow1(s * rstd * Storage<DT>::widen1(weight[j]));
+            }
+        }
     }
 }
 
 // ---------------------------------------------------------------------------------------------
-// Kernel 3: silu_and_mul, one thread per element (design 0) or per element pair (design 1).
+// Kernel 3: silu_and_mul, grid-stride over the outputs.  FAST = false: one 16-bit element per
+// access, the library exponential and a true division.  FAST = true: two elements per 32-bit
+// access, the fast exponential and a reciprocal-multiply in place of the division (the intrinsics
+// Section 5.3 names); for gates below about -88 the exponential overflows and the result is -0,
+// as with the division.
 // ---------------------------------------------------------------------------------------------
-template <int DT>
-__global__ void __launch_bounds__(kThreads)
-silu_scalar_kernel(uint16_t *out, const uint16_t *in, int64_t total, int64_t D) {
-    const int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
-    if (i >= total) return;
-    const int64_t row = i / D, col = i - row * D;
-    const float a = Storage<DT>::widen1(in[row * 2 * D + col]);
-    const float b = Storage<DT>::widen1(in[row * 2 * D + D + col]);
-    out[i] = Storage<DT>::narrow1(a / (1.0f + expf(-a)) * b);  // library exponential and a division
+template <bool FAST>
+__device__ __forceinline__ float gated(float a, float b) {
+    if constexpr (FAST) {
+        const float sigmoid = __frcp_rn(1.0f + __expf(-a));
+        return a * sigmoid * b;
+    } else {
+        return a / (1.0f + expf(-a)) * b;
+    }
 }
 
-__device__ __forceinline__ float silu_fast(float a) {
-    // fast exponential, then reciprocal and multiply in place of the division (as described; for
-    // gates below about -88 the exponential overflows and the result is -0, like design 0)
-    const float e = __expf(-a);
-    return __fmul_rn(a, __frcp_rn(1.0f + e));
+template <int DT, bool FAST, int BLOCK>
+__global__ void __launch_bounds__(BLOCK)
+silu_pair_kernel(uint16_t *out, const uint16_t *in, int64_t T, int64_t D) {
+    const int64_t per_row = FAST ? D / 2 : D;  // work items per row: element pairs or elements
+    const int64_t items = T * per_row;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * BLOCK;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * BLOCK + threadIdx.x; i < items; i += stride) {
+        const int64_t row = i / per_row, col = i - row * per_row;
+        if constexpr (FAST) {
+            const uint32_t *in2 = reinterpret_cast<const uint32_t *>(in) + row * 2 * per_row;
+            float a_lo, a_hi, b_lo, b_hi;
+            Storage<DT>::widen2(in2[col], a_lo, a_hi);
+            Storage<DT>::widen2(in2[per_row + col], b_lo, b_hi);
+            reinterpret_cast<uint32_t *>(out)[i] = Storage<DT>::narrow2(gated<true>(a_lo, b_lo), gated<true>(a_hi, b_hi));
+        } else {
+            const uint16_t *gate = in + row * 2 * D;
+            out[i] = Storage<DT>::narrow1(gated<false>(Storage<DT>::widen1(gate[col]), Storage<DT>::widen1(gate[D + col])));
+        }
+    }
 }
 
-template <int DT>
-__global__ void __launch_bounds__(kThreads)
-silu_pair_kernel(uint16_t *out, const uint16_t *in, int64_t total_pairs, int64_t halfD) {
-    const int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
-    if (i >= total_pairs) return;
-    const int64_t row = i / halfD, col = i - row * halfD;
-    const uint32_t *pin = reinterpret_cast<const uint32_t *>(in);
-    float a0, a1, b0, b1;
-    Storage<DT>::widen2(pin[row * 2 * halfD + col], a0, a1);
-    Storage<DT>::widen2(pin[row * 2 * halfD + halfD + col], b0, b1);
-    reinterpret_cast<uint32_t *>(out)[i] = Storage<DT>::narrow2(__fmul_rn(silu_fast(a0), b0), __fmul_rn(silu_fast(a1), b1));
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+inline bool word_aligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 3) == 0; }
+
+// Blocks for `work` block-sized pieces: all of them, up to a few waves per SM (the kernels stride).
+inline unsigned grid_for(int64_t work) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        sms = 148;
+    const int64_t cap = static_cast<int64_t>(sms) * kWavesOfBlocks * (2048 / kBlock);
+    return static_cast<unsigned>(work < cap ? (work < 1 ? 1 : work) : cap);
 }
 
-inline bool aligned4(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 3) == 0; }
-inline astra_status_t launched() { return cudaGetLastError() == cudaSuccess ? ASTRA_OK : ASTRA_ERR_CUDA; }
+template <typename... KArgs, typename... Args>
+inline astra_status_t run(void (*kernel)(KArgs...), unsigned grid, cudaStream_t stream, Args... args) {
+    kernel<<<grid, kBlock, 0, stream>>>(static_cast<KArgs>(args)...);
+    return cudaGetLastError() == cudaSuccess ? ASTRA_OK : ASTRA_ERR_CUDA;
+}
+
+// Runs CALL with DT bound to the (validated, 16-bit) dtype and VARIANT to the design.
+#define ABLATION_DISPATCH(dtype, design, CALL)                                            \
+    do {                                                                                  \
+        if ((dtype) == ASTRA_BF16) {                                                      \
+            constexpr int DT = ASTRA_BF16;                                                \
+            if (design) { constexpr bool VARIANT = true; return CALL; }                   \
+            constexpr bool VARIANT = false; return CALL;                                  \
+        }                                                                                 \
+        constexpr int DT = ASTRA_FP16;                                                    \
+        if (design) { constexpr bool VARIANT = true; return CALL; }                       \
+        constexpr bool VARIANT = false; return CALL;                                      \
+    } while (0)
 
 }  // namespace
 
@@ -196,24 +259,16 @@ astra_status_t astra_ablation_merge_attn_states_lse(int design, void *v_out, flo
     if (design != 0 && design != 1) return ASTRA_ERR_BAD_SHAPE;
     if (T < 0 || Hh <= 0 || D <= 0 || D > 65536 || (design == 1 && D % 2)) return ASTRA_ERR_BAD_SHAPE;
     if (T > 0 && Hh > (1ll << 40) / T) return ASTRA_ERR_BAD_SHAPE;
-    if (design == 1 && !(aligned4(v_out) && aligned4(v_a) && aligned4(v_b))) return ASTRA_ERR_MISALIGNED;
+    if (design == 1 && !(word_aligned(v_out) && word_aligned(v_a) && word_aligned(v_b))) return ASTRA_ERR_MISALIGNED;
     if (T == 0) return ASTRA_OK;
     const int64_t rows = T * Hh;
-    const int64_t blocks = (rows + kThreads / 32 - 1) / (kThreads / 32);
-    if (blocks > 2147483647ll) return ASTRA_ERR_BAD_SHAPE;
+    const unsigned grid = grid_for((rows + kBlock / 32 - 1) / (kBlock / 32));
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     uint16_t *vo = static_cast<uint16_t *>(v_out);
     const uint16_t *va = static_cast<const uint16_t *>(v_a), *vb = static_cast<const uint16_t *>(v_b);
-    const unsigned g = static_cast<unsigned>(blocks);
-    const int d = static_cast<int>(D);
-    if (design == 0) {
-        if (dtype == ASTRA_BF16) merge_recompute_kernel<ASTRA_BF16><<<g, kThreads, 0, st>>>(vo, lse_out, va, lse_a, vb, lse_b, rows, d);
-        else merge_recompute_kernel<ASTRA_FP16><<<g, kThreads, 0, st>>>(vo, lse_out, va, lse_a, vb, lse_b, rows, d);
-    } else {
-        if (dtype == ASTRA_BF16) merge_hoisted_kernel<ASTRA_BF16><<<g, kThreads, 0, st>>>(vo, lse_out, va, lse_a, vb, lse_b, rows, d);
-        else merge_hoisted_kernel<ASTRA_FP16><<<g, kThreads, 0, st>>>(vo, lse_out, va, lse_a, vb, lse_b, rows, d);
-    }
-    return launched();
+    ABLATION_DISPATCH(dtype, design,
+                      run(merge_pair_kernel<DT, VARIANT, kBlock>, grid, st, vo, lse_out, va, lse_a, vb, lse_b, rows,
+                          static_cast<int>(D)));
 }
 
 astra_status_t astra_ablation_fused_add_rmsnorm(int design, void *x, void *residual, const void *weight,
@@ -223,21 +278,14 @@ astra_status_t astra_ablation_fused_add_rmsnorm(int design, void *x, void *resid
     if (dtype != ASTRA_BF16 && dtype != ASTRA_FP16) return ASTRA_ERR_BAD_DTYPE;
     if (design != 0 && design != 1) return ASTRA_ERR_BAD_SHAPE;
     if (T < 0 || T > 2147483647ll || H <= 0 || H > 65536 || (design == 1 && H % 2)) return ASTRA_ERR_BAD_SHAPE;
-    if (design == 1 && !(aligned4(x) && aligned4(residual) && aligned4(weight))) return ASTRA_ERR_MISALIGNED;
+    if (design == 1 && !(word_aligned(x) && word_aligned(residual) && word_aligned(weight))) return ASTRA_ERR_MISALIGNED;
     if (T == 0) return ASTRA_OK;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     uint16_t *xp = static_cast<uint16_t *>(x), *rp = static_cast<uint16_t *>(residual);
     const uint16_t *wp = static_cast<const uint16_t *>(weight);
-    const unsigned g = static_cast<unsigned>(T);
-    const int h = static_cast<int>(H);
-    if (design == 0) {
-        if (dtype == ASTRA_BF16) rmsnorm_tree_kernel<ASTRA_BF16><<<g, kThreads, 0, st>>>(xp, rp, wp, h, eps);
-        else rmsnorm_tree_kernel<ASTRA_FP16><<<g, kThreads, 0, st>>>(xp, rp, wp, h, eps);
-    } else {
-        if (dtype == ASTRA_BF16) rmsnorm_shuffle_kernel<ASTRA_BF16><<<g, kThreads, 0, st>>>(xp, rp, wp, h, eps);
-        else rmsnorm_shuffle_kernel<ASTRA_FP16><<<g, kThreads, 0, st>>>(xp, rp, wp, h, eps);
-    }
-    return launched();
+    const unsigned grid = static_cast<unsigned>(T);  // one block per row (the stride loop then runs once)
+    ABLATION_DISPATCH(dtype, design,
+                      run(rmsnorm_pair_kernel<DT, VARIANT, kBlock>, grid, st, xp, rp, wp, T, static_cast<int>(H), eps));
 }
 
 astra_status_t astra_ablation_silu_and_mul(int design, void *out, const void *input, int64_t T, int64_t D,
@@ -247,23 +295,14 @@ astra_status_t astra_ablation_silu_and_mul(int design, void *out, const void *in
     if (design != 0 && design != 1) return ASTRA_ERR_BAD_SHAPE;
     if (T < 0 || D <= 0 || D > (1ll << 30) || (design == 1 && D % 2)) return ASTRA_ERR_BAD_SHAPE;
     if (T > 0 && D > (1ll << 38) / T) return ASTRA_ERR_BAD_SHAPE;
-    if (design == 1 && !(aligned4(out) && aligned4(input))) return ASTRA_ERR_MISALIGNED;
+    if (design == 1 && !(word_aligned(out) && word_aligned(input))) return ASTRA_ERR_MISALIGNED;
     if (T == 0) return ASTRA_OK;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     uint16_t *op = static_cast<uint16_t *>(out);
     const uint16_t *ip = static_cast<const uint16_t *>(input);
-    const int64_t total = (design == 0) ? T * D : T * (D / 2);
-    const int64_t blocks = (total + kThreads - 1) / kThreads;
-    if (blocks > 2147483647ll) return ASTRA_ERR_BAD_SHAPE;
-    const unsigned g = static_cast<unsigned>(blocks);
-    if (design == 0) {
-        if (dtype == ASTRA_BF16) silu_scalar_kernel<ASTRA_BF16><<<g, kThreads, 0, st>>>(op, ip, total, D);
-        else silu_scalar_kernel<ASTRA_FP16><<<g, kThreads, 0, st>>>(op, ip, total, D);
-    } else {
-        if (dtype == ASTRA_BF16) silu_pair_kernel<ASTRA_BF16><<<g, kThreads, 0, st>>>(op, ip, total, D / 2);
-        else silu_pair_kernel<ASTRA_FP16><<<g, kThreads, 0, st>>>(op, ip, total, D / 2);
-    }
-    return launched();
+    const int64_t items = design == 0 ? T * D : T * (D / 2);
+    const unsigned grid = grid_for((items + kBlock - 1) / kBlock);
+    ABLATION_DISPATCH(dtype, design, run(silu_pair_kernel<DT, VARIANT, kBlock>, grid, st, op, ip, T, D));
 }
 
 }  // extern "C"

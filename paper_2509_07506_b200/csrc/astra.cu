@@ -1,6 +1,9 @@
 // C ABI of the library (declared in astra.h): argument validation, launch-shape selection per
 // width / alignment / row count, and the kernel launches.  Nothing here allocates, synchronises or
-// keeps state; every failure is reported as a status code before anything is launched.
+// keeps state.  Argument errors are reported before anything is launched; a launch the runtime
+// refuses is reported as ASTRA_ERR_CUDA from that launch's own return value (the thread's sticky
+// "last error" of the CUDA runtime is neither read nor cleared on the success path), and the
+// remaining launches of a split call are not issued.
 #include <cuda_runtime.h>
 
 #include "astra.h"
@@ -8,9 +11,17 @@
 #include "merge_attn_states_lse.cuh"
 #include "silu_and_mul.cuh"
 
+#ifndef ASTRA_BUILD_ID
+#define ASTRA_BUILD_ID "unidentified"
+#endif
+
 namespace {
 
 using namespace astra;
+
+// Hash of the sources this library was compiled from (set by the build script), behind a marker
+// that can also be found in the file without loading it.
+const char kBuildId[] = "astra-build-id:" ASTRA_BUILD_ID;
 
 inline bool aligned(const void *p, size_t bytes) {
     return (reinterpret_cast<uintptr_t>(p) % bytes) == 0;
@@ -59,8 +70,13 @@ struct VecPick {
     }
 };
 
-inline astra_status_t launch_status() {
-    return cudaGetLastError() == cudaSuccess ? ASTRA_OK : ASTRA_ERR_CUDA;
+// Status of a call from the result of its launch(es).  After a refused launch the runtime's
+// per-thread last-error slot holds that refusal; it has been reported through the return code, so it
+// is taken out again rather than left to surface in some later, unrelated check of the caller's.
+inline astra_status_t launch_status(cudaError_t err) {
+    if (err == cudaSuccess) return ASTRA_OK;
+    (void)cudaGetLastError();
+    return ASTRA_ERR_CUDA;
 }
 
 // Every kernel is launched with programmatic stream serialization allowed: its blocks may be
@@ -68,8 +84,8 @@ inline astra_status_t launch_status() {
 // for that kernel to complete before their first global access.  Stream order is unchanged; the
 // launch latency and block prologue of back-to-back calls overlap the previous kernel's tail.
 template <typename... KArgs, typename... Args>
-inline void launch(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t stream,
-                   Args... args) {
+inline cudaError_t launch(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t stream,
+                          Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(block);
@@ -80,7 +96,7 @@ inline void launch(void (*kernel)(KArgs...), unsigned grid, unsigned block, cuda
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);  // failure is read back by launch_status()
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 // Flat vector indices are 31-bit and grids are limited to 2^31-1 blocks; larger inputs are split
@@ -100,8 +116,8 @@ inline void launch(void (*kernel)(KArgs...), unsigned grid, unsigned block, cuda
 // The same, for a kernel whose consecutive groups of `cluster` blocks form thread-block clusters
 // (distributed shared memory between the blocks of a group).
 template <typename... KArgs, typename... Args>
-inline void launch_clustered(void (*kernel)(KArgs...), unsigned grid, unsigned block, unsigned cluster,
-                             cudaStream_t stream, Args... args) {
+inline cudaError_t launch_clustered(void (*kernel)(KArgs...), unsigned grid, unsigned block, unsigned cluster,
+                                    cudaStream_t stream, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(block);
@@ -116,11 +132,15 @@ inline void launch_clustered(void (*kernel)(KArgs...), unsigned grid, unsigned b
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 constexpr int64_t kMaxVecsPerLaunch = ASTRA_MAX_VECS_PER_LAUNCH;
 constexpr int64_t kInt64Max = 9223372036854775807ll;
+// Widest row of fused_add_rmsnorm, in 16-bit units (2^30 bf16/fp16 or 2^29 fp32 elements, a 2 GiB
+// row): unit offsets inside a row, and the rounded-up vector counts derived from them, then fit a
+// 32-bit signed integer.
+constexpr int64_t kMaxRowUnits = 1ll << 30;
 
 inline bool valid_dtype(astra_dtype_t d) { return d == ASTRA_BF16 || d == ASTRA_FP16 || d == ASTRA_FP32; }
 
@@ -142,8 +162,8 @@ inline int64_t units_per_elem(astra_dtype_t d) { return d == ASTRA_FP32 ? 2 : 1;
 // ---------------------------------------------------------------------------------------------
 // D, the pitches and the pointers are in 16-bit units; UVEC is the vector width in units.
 template <int DT, int UVEC, int UNROLL, int THREADS>
-void launch_silu(uint16_t *out, const uint16_t *gate, const uint16_t *up, int64_t T, int64_t D,
-                 int64_t out_pitch, int64_t gate_pitch, int64_t up_pitch, cudaStream_t stream) {
+cudaError_t launch_silu(uint16_t *out, const uint16_t *gate, const uint16_t *up, int64_t T, int64_t D,
+                        int64_t out_pitch, int64_t gate_pitch, int64_t up_pitch, cudaStream_t stream) {
   if constexpr (UVEC >= Storage<DT>::UNITS) {
     constexpr int VEC = UVEC / Storage<DT>::UNITS;
     const int64_t nvec = D / UVEC;
@@ -153,50 +173,53 @@ void launch_silu(uint16_t *out, const uint16_t *gate, const uint16_t *up, int64_
         const uint32_t total = static_cast<uint32_t>(rows * nvec);
         const uint32_t tile = THREADS * UNROLL;
         const uint32_t blocks = (total + tile - 1) / tile;
-        launch(silu_and_mul_kernel<DT, VEC, UNROLL, THREADS>, blocks, THREADS, stream,
-               out + t0 * out_pitch, gate + t0 * gate_pitch, up + t0 * up_pitch, total,
-               FastDiv::make(static_cast<uint32_t>(nvec)), out_pitch, gate_pitch, up_pitch);
+        const cudaError_t err = launch(silu_and_mul_kernel<DT, VEC, UNROLL, THREADS>, blocks, THREADS, stream,
+                                       out + t0 * out_pitch, gate + t0 * gate_pitch, up + t0 * up_pitch, total,
+                                       FastDiv::make(static_cast<uint32_t>(nvec)), out_pitch, gate_pitch, up_pitch);
+        if (err != cudaSuccess) return err;
     }
   }
+  return cudaSuccess;
 }
 
 template <int DT>
-void dispatch_silu(uint16_t *out, const uint16_t *gate, const uint16_t *up, int64_t T, int64_t D,
+cudaError_t dispatch_silu(uint16_t *out, const uint16_t *gate, const uint16_t *up, int64_t T, int64_t D,
                    int64_t out_pitch, int64_t gate_pitch, int64_t up_pitch, cudaStream_t stream) {
     const int vec = VecPick(8).extent(D).extent(out_pitch).extent(gate_pitch).extent(up_pitch)
                         .pointer(out).pointer(gate).pointer(up).vec;
     // One 16-byte vector per thread and 256-thread blocks: the smallest work quantum that still
     // keeps the block scheduler ahead, which gives the shortest drain at the end of the grid.
     switch (vec) {
-        case 8: launch_silu<DT, 8, 1, 256>(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, stream); break;
-        case 4: launch_silu<DT, 4, 4, 256>(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, stream); break;
-        case 2: launch_silu<DT, 2, 4, 256>(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, stream); break;
-        default: launch_silu<DT, 1, 4, 256>(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, stream); break;
+        case 8: return launch_silu<DT, 8, 1, 256>(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, stream);
+        case 4: return launch_silu<DT, 4, 4, 256>(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, stream);
+        case 2: return launch_silu<DT, 2, 4, 256>(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, stream);
+        default: return launch_silu<DT, 1, 4, 256>(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, stream);
     }
 }
 
 astra_status_t silu_entry(void *out, const void *gate, const void *up, int64_t T, int64_t D,
                           int64_t out_pitch, int64_t gate_pitch, int64_t up_pitch,
                           astra_dtype_t dtype, void *cuda_stream) {
-    if (!out || !gate || !up) return ASTRA_ERR_NULL_POINTER;
     if (!valid_dtype(dtype)) return ASTRA_ERR_BAD_DTYPE;
     if (T < 0 || D <= 0 || D > 1073741823ll) return ASTRA_ERR_BAD_SHAPE;
     if (out_pitch < D || gate_pitch < D || up_pitch < D) return ASTRA_ERR_BAD_SHAPE;
     const int64_t max_pitch = out_pitch > gate_pitch ? (out_pitch > up_pitch ? out_pitch : up_pitch)
                                                      : (gate_pitch > up_pitch ? gate_pitch : up_pitch);
     if (T > 0 && max_pitch > kInt64Max / 4 / T) return ASTRA_ERR_BAD_SHAPE;
+    if (T == 0) return ASTRA_OK;  // an empty batch has no data to point at: its pointers are not examined
+    if (!out || !gate || !up) return ASTRA_ERR_NULL_POINTER;
     const int64_t U = units_per_elem(dtype);
     const size_t eb = static_cast<size_t>(2 * U);
     if (!aligned(out, eb) || !aligned(gate, eb) || !aligned(up, eb)) return ASTRA_ERR_MISALIGNED;
-    if (T == 0) return ASTRA_OK;
     const int64_t Du = D * U, opu = out_pitch * U, gpu = gate_pitch * U, upu = up_pitch * U;  // in units
     if (pitched_overlap(out, opu, gate, gpu, T, Du) || pitched_overlap(out, opu, up, upu, T, Du))
         return ASTRA_ERR_OVERLAP;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     uint16_t *op = static_cast<uint16_t *>(out);
     const uint16_t *gp = static_cast<const uint16_t *>(gate), *upp = static_cast<const uint16_t *>(up);
-    ASTRA_FOR_DTYPE(dtype, dispatch_silu<DT>(op, gp, upp, T, Du, opu, gpu, upu, stream));
-    return launch_status();
+    cudaError_t err = cudaSuccess;
+    ASTRA_FOR_DTYPE(dtype, err = dispatch_silu<DT>(op, gp, upp, T, Du, opu, gpu, upu, stream));
+    return launch_status(err);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -204,7 +227,7 @@ astra_status_t silu_entry(void *out, const void *gate, const void *up, int64_t T
 // ---------------------------------------------------------------------------------------------
 // D and the value pointers are in 16-bit units; UVEC is the vector width in units.
 template <int DT, int UVEC, int UNROLL, int THREADS>
-void launch_merge(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
+cudaError_t launch_merge(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
                   const uint16_t *v_b, const float *lse_b, int64_t rows_total, int64_t D,
                   cudaStream_t stream) {
   if constexpr (UVEC >= Storage<DT>::UNITS) {
@@ -216,29 +239,32 @@ void launch_merge(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const fl
         const uint32_t total = static_cast<uint32_t>(rows * nvec);
         const uint32_t tile = THREADS * UNROLL;
         const uint32_t blocks = (total + tile - 1) / tile;
-        launch(merge_attn_states_lse_kernel<DT, VEC, UNROLL, THREADS>, blocks, THREADS, stream,
-               v_out + r0 * D, lse_out ? lse_out + r0 : nullptr, v_a + r0 * D, lse_a + r0, v_b + r0 * D,
-               lse_b + r0, total, FastDiv::make(static_cast<uint32_t>(nvec)));
+        const cudaError_t err =
+            launch(merge_attn_states_lse_kernel<DT, VEC, UNROLL, THREADS>, blocks, THREADS, stream,
+                   v_out + r0 * D, lse_out ? lse_out + r0 : nullptr, v_a + r0 * D, lse_a + r0, v_b + r0 * D,
+                   lse_b + r0, total, FastDiv::make(static_cast<uint32_t>(nvec)));
+        if (err != cudaSuccess) return err;
     }
   }
+  return cudaSuccess;
 }
 
 template <int DT>
-void dispatch_merge(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
+cudaError_t dispatch_merge(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
                     const uint16_t *v_b, const float *lse_b, int64_t rows, int64_t D,
                     cudaStream_t stream) {
     // 32-byte accesses measured best here (one per thread, 256-thread blocks)
     switch (VecPick(16).extent(D).pointer(v_out).pointer(v_a).pointer(v_b).vec) {
-        case 16: launch_merge<DT, 16, 1, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream); break;
-        case 8: launch_merge<DT, 8, 2, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream); break;
-        case 4: launch_merge<DT, 4, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream); break;
-        case 2: launch_merge<DT, 2, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream); break;
-        default: launch_merge<DT, 1, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream); break;
+        case 16: return launch_merge<DT, 16, 1, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream);
+        case 8: return launch_merge<DT, 8, 2, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream);
+        case 4: return launch_merge<DT, 4, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream);
+        case 2: return launch_merge<DT, 2, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream);
+        default: return launch_merge<DT, 1, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, D, stream);
     }
 }
 
 template <int DT, int UVEC, int UNROLL, int THREADS>
-void launch_merge_strided(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
+cudaError_t launch_merge_strided(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
                           const uint16_t *v_b, const float *lse_b, int64_t rows_total, int64_t Hh,
                           int64_t D, const MergeStrides &st, cudaStream_t stream) {
   if constexpr (UVEC >= Storage<DT>::UNITS) {
@@ -250,25 +276,28 @@ void launch_merge_strided(uint16_t *v_out, float *lse_out, const uint16_t *v_a, 
         const uint32_t total = static_cast<uint32_t>(rows * nvec);
         const uint32_t tile = THREADS * UNROLL;
         const uint32_t blocks = (total + tile - 1) / tile;
-        launch(merge_attn_states_lse_strided_kernel<DT, VEC, UNROLL, THREADS>, blocks, THREADS, stream,
-               v_out, lse_out, v_a, lse_a, v_b, lse_b, total, static_cast<uint32_t>(r0),
-               FastDiv::make(static_cast<uint32_t>(nvec)), FastDiv::make(static_cast<uint32_t>(Hh)), st);
+        const cudaError_t err =
+            launch(merge_attn_states_lse_strided_kernel<DT, VEC, UNROLL, THREADS>, blocks, THREADS, stream,
+                   v_out, lse_out, v_a, lse_a, v_b, lse_b, total, static_cast<uint32_t>(r0),
+                   FastDiv::make(static_cast<uint32_t>(nvec)), FastDiv::make(static_cast<uint32_t>(Hh)), st);
+        if (err != cudaSuccess) return err;
     }
   }
+  return cudaSuccess;
 }
 
 template <int DT>
-void dispatch_merge_strided(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
+cudaError_t dispatch_merge_strided(uint16_t *v_out, float *lse_out, const uint16_t *v_a, const float *lse_a,
                             const uint16_t *v_b, const float *lse_b, int64_t rows, int64_t Hh, int64_t D,
                             const MergeStrides &st, cudaStream_t stream) {
     const int vec = VecPick(16).extent(D).extent(st.va_t).extent(st.va_h).extent(st.vb_t).extent(st.vb_h)
                         .extent(st.vo_t).extent(st.vo_h).pointer(v_out).pointer(v_a).pointer(v_b).vec;
     switch (vec) {
-        case 16: launch_merge_strided<DT, 16, 1, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, Hh, D, st, stream); break;
-        case 8: launch_merge_strided<DT, 8, 2, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, Hh, D, st, stream); break;
-        case 4: launch_merge_strided<DT, 4, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, Hh, D, st, stream); break;
-        case 2: launch_merge_strided<DT, 2, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, Hh, D, st, stream); break;
-        default: launch_merge_strided<DT, 1, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, Hh, D, st, stream); break;
+        case 16: return launch_merge_strided<DT, 16, 1, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, Hh, D, st, stream);
+        case 8: return launch_merge_strided<DT, 8, 2, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, Hh, D, st, stream);
+        case 4: return launch_merge_strided<DT, 4, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, Hh, D, st, stream);
+        case 2: return launch_merge_strided<DT, 2, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, Hh, D, st, stream);
+        default: return launch_merge_strided<DT, 1, 4, 256>(v_out, lse_out, v_a, lse_a, v_b, lse_b, rows, Hh, D, st, stream);
     }
 }
 
@@ -303,12 +332,13 @@ constexpr int rmsnorm_max_units_per_thread(int uvec) { return uvec == 1 ? 8 : 64
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 template <int DT, int UVEC, int VPT>
-inline void launch_rmsnorm_reg(unsigned rows, int threads, cudaStream_t stream, const RmsnormOperands &op,
-                               const uint16_t *w, int H, float eps, float inv_H) {
+inline cudaError_t launch_rmsnorm_reg(unsigned rows, int threads, cudaStream_t stream, const RmsnormOperands &op,
+                                      const uint16_t *w, int H, float eps, float inv_H) {
     // wider combinations than the per-thread cap are never selected and are not instantiated
     if constexpr (UVEC * VPT <= rmsnorm_max_units_per_thread(UVEC))
-        launch(fused_add_rmsnorm_reg_kernel<DT, UVEC / Storage<DT>::UNITS, VPT>, rows, threads, stream, op, w, H,
-               eps, inv_H);
+        return launch(fused_add_rmsnorm_reg_kernel<DT, UVEC / Storage<DT>::UNITS, VPT>, rows, threads, stream, op,
+                      w, H, eps, inv_H);
+    return cudaErrorInvalidValue;
 }
 
 // Register-resident rows: VPT vectors per thread with blockDim = ceil(nvec / VPT) rounded up to a warp.
@@ -318,7 +348,7 @@ inline void launch_rmsnorm_reg(unsigned rows, int threads, cudaStream_t stream, 
 // H is in elements; the operands' pointers and pitches are in 16-bit units; UVEC is the vector width
 // in units.
 template <int DT, int UVEC>
-void launch_rmsnorm(RmsnormOperands op, const uint16_t *w, int64_t T, int H, float eps, cudaStream_t stream) {
+cudaError_t launch_rmsnorm(RmsnormOperands op, const uint16_t *w, int64_t T, int H, float eps, cudaStream_t stream) {
   if constexpr (UVEC >= Storage<DT>::UNITS) {
     constexpr int VEC = UVEC / Storage<DT>::UNITS;
     constexpr int kMaxVpt = rmsnorm_max_units_per_thread(UVEC) / UVEC;
@@ -357,40 +387,41 @@ void launch_rmsnorm(RmsnormOperands op, const uint16_t *w, int64_t T, int H, flo
         o.r += t0 * op.r_pitch;
         o.y += t0 * op.y_pitch;
         o.r_out += t0 * op.r_out_pitch;
+        cudaError_t err = cudaSuccess;
         if (cluster) {
             if constexpr (UVEC >= 4)
-                launch_clustered(fused_add_rmsnorm_cluster_kernel<DT, VEC, kClusterVpt>, rows * cluster,
-                                 cluster_threads, cluster, stream, o, w, H, eps, inv_H);
-            continue;
+                err = launch_clustered(fused_add_rmsnorm_cluster_kernel<DT, VEC, kClusterVpt>, rows * cluster,
+                                       cluster_threads, cluster, stream, o, w, H, eps, inv_H);
+        } else if (!fits) {
+            err = launch(fused_add_rmsnorm_twopass_kernel<DT, VEC>, rows, sweep_threads, stream, o, w, H, eps, inv_H);
+        } else {
+            switch (vpt) {
+                case 1: err = launch_rmsnorm_reg<DT, UVEC, 1>(rows, threads, stream, o, w, H, eps, inv_H); break;
+                case 2: err = launch_rmsnorm_reg<DT, UVEC, 2>(rows, threads, stream, o, w, H, eps, inv_H); break;
+                case 4: err = launch_rmsnorm_reg<DT, UVEC, 4>(rows, threads, stream, o, w, H, eps, inv_H); break;
+                case 8: err = launch_rmsnorm_reg<DT, UVEC, 8>(rows, threads, stream, o, w, H, eps, inv_H); break;
+                case 16: err = launch_rmsnorm_reg<DT, UVEC, 16>(rows, threads, stream, o, w, H, eps, inv_H); break;
+                case 32: err = launch_rmsnorm_reg<DT, UVEC, 32>(rows, threads, stream, o, w, H, eps, inv_H); break;
+                default: err = launch_rmsnorm_reg<DT, UVEC, 64>(rows, threads, stream, o, w, H, eps, inv_H); break;
+            }
         }
-        if (!fits) {
-            launch(fused_add_rmsnorm_twopass_kernel<DT, VEC>, rows, sweep_threads, stream, o, w, H, eps, inv_H);
-            continue;
-        }
-        switch (vpt) {
-            case 1: launch_rmsnorm_reg<DT, UVEC, 1>(rows, threads, stream, o, w, H, eps, inv_H); break;
-            case 2: launch_rmsnorm_reg<DT, UVEC, 2>(rows, threads, stream, o, w, H, eps, inv_H); break;
-            case 4: launch_rmsnorm_reg<DT, UVEC, 4>(rows, threads, stream, o, w, H, eps, inv_H); break;
-            case 8: launch_rmsnorm_reg<DT, UVEC, 8>(rows, threads, stream, o, w, H, eps, inv_H); break;
-            case 16: launch_rmsnorm_reg<DT, UVEC, 16>(rows, threads, stream, o, w, H, eps, inv_H); break;
-            case 32: launch_rmsnorm_reg<DT, UVEC, 32>(rows, threads, stream, o, w, H, eps, inv_H); break;
-            default: launch_rmsnorm_reg<DT, UVEC, 64>(rows, threads, stream, o, w, H, eps, inv_H); break;
-        }
+        if (err != cudaSuccess) return err;
     }
   }
+  return cudaSuccess;
 }
 
 template <int DT>
-void dispatch_rmsnorm(const RmsnormOperands &op, const uint16_t *w, int64_t T, int H, float eps,
+cudaError_t dispatch_rmsnorm(const RmsnormOperands &op, const uint16_t *w, int64_t T, int H, float eps,
                       cudaStream_t stream) {
     const int vec = VecPick(8).extent(static_cast<int64_t>(H) * Storage<DT>::UNITS).extent(op.x_pitch)
                         .extent(op.r_pitch).extent(op.y_pitch).extent(op.r_out_pitch).pointer(op.x)
                         .pointer(op.r).pointer(op.y).pointer(op.r_out).pointer(w).vec;
     switch (vec) {
-        case 8: launch_rmsnorm<DT, 8>(op, w, T, H, eps, stream); break;
-        case 4: launch_rmsnorm<DT, 4>(op, w, T, H, eps, stream); break;
-        case 2: launch_rmsnorm<DT, 2>(op, w, T, H, eps, stream); break;
-        default: launch_rmsnorm<DT, 1>(op, w, T, H, eps, stream); break;
+        case 8: return launch_rmsnorm<DT, 8>(op, w, T, H, eps, stream);
+        case 4: return launch_rmsnorm<DT, 4>(op, w, T, H, eps, stream);
+        case 2: return launch_rmsnorm<DT, 2>(op, w, T, H, eps, stream);
+        default: return launch_rmsnorm<DT, 1>(op, w, T, H, eps, stream);
     }
 }
 
@@ -398,21 +429,22 @@ astra_status_t rmsnorm_entry(void *y, void *residual_out, const void *x, const v
                              const void *weight, int64_t T, int64_t H, int64_t y_pitch,
                              int64_t ro_pitch, int64_t x_pitch, int64_t r_pitch, float eps,
                              astra_dtype_t dtype, void *cuda_stream) {
-    if (!y || !residual_out || !x || !residual || !weight) return ASTRA_ERR_NULL_POINTER;
     if (!valid_dtype(dtype)) return ASTRA_ERR_BAD_DTYPE;
-    if (T < 0 || H <= 0 || H > 2147483647ll) return ASTRA_ERR_BAD_SHAPE;
+    const int64_t U = units_per_elem(dtype);
+    // a row is indexed in 16-bit units with 32-bit integers inside the kernels
+    if (T < 0 || H <= 0 || H > kMaxRowUnits / U) return ASTRA_ERR_BAD_SHAPE;
     if (y_pitch < H || ro_pitch < H || x_pitch < H || r_pitch < H) return ASTRA_ERR_BAD_SHAPE;
     int64_t max_pitch = y_pitch;
     if (ro_pitch > max_pitch) max_pitch = ro_pitch;
     if (x_pitch > max_pitch) max_pitch = x_pitch;
     if (r_pitch > max_pitch) max_pitch = r_pitch;
     if (T > 0 && max_pitch > kInt64Max / 4 / T) return ASTRA_ERR_BAD_SHAPE;
-    const int64_t U = units_per_elem(dtype);
+    if (T == 0) return ASTRA_OK;
+    if (!y || !residual_out || !x || !residual || !weight) return ASTRA_ERR_NULL_POINTER;
     const size_t eb = static_cast<size_t>(2 * U);
     if (!aligned(y, eb) || !aligned(residual_out, eb) || !aligned(x, eb) || !aligned(residual, eb) ||
         !aligned(weight, eb))
         return ASTRA_ERR_MISALIGNED;
-    if (T == 0) return ASTRA_OK;
     // from here on widths and pitches are in 16-bit units
     const int64_t Hu = H * U;
     y_pitch *= U;
@@ -441,8 +473,9 @@ astra_status_t rmsnorm_entry(void *y, void *residual_out, const void *x, const v
     op.r_out_pitch = ro_pitch;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const uint16_t *wp = static_cast<const uint16_t *>(weight);
-    ASTRA_FOR_DTYPE(dtype, dispatch_rmsnorm<DT>(op, wp, T, static_cast<int>(H), eps, stream));
-    return launch_status();
+    cudaError_t err = cudaSuccess;
+    ASTRA_FOR_DTYPE(dtype, err = dispatch_rmsnorm<DT>(op, wp, T, static_cast<int>(H), eps, stream));
+    return launch_status(err);
 }
 
 }  // namespace
@@ -465,8 +498,10 @@ astra_status_t astra_fused_add_rmsnorm_ex(void *y, void *residual_out, const voi
 
 astra_status_t astra_silu_and_mul(void *out, const void *input, int64_t T, int64_t D,
                                   astra_dtype_t dtype, void *cuda_stream) {
+    if (!valid_dtype(dtype)) return ASTRA_ERR_BAD_DTYPE;
+    if (T < 0 || D <= 0 || D > 1073741823ll) return ASTRA_ERR_BAD_SHAPE;
+    if (T == 0) return ASTRA_OK;
     if (!input) return ASTRA_ERR_NULL_POINTER;
-    if (D <= 0 || D > 1073741823ll) return ASTRA_ERR_BAD_SHAPE;
     const void *up = static_cast<const uint16_t *>(input) + D * units_per_elem(dtype);
     return silu_entry(out, input, up, T, D, D, 2 * D, 2 * D, dtype, cuda_stream);
 }
@@ -481,16 +516,16 @@ astra_status_t astra_merge_attn_states_lse(void *v_out, float *lse_out, const vo
                                            const float *lse_a, const void *v_b, const float *lse_b,
                                            int64_t T, int64_t Hh, int64_t D, astra_dtype_t dtype,
                                            void *cuda_stream) {
-    if (!v_out || !v_a || !v_b || !lse_a || !lse_b) return ASTRA_ERR_NULL_POINTER;
     if (!valid_dtype(dtype)) return ASTRA_ERR_BAD_DTYPE;
-    if (T < 0 || Hh <= 0 || D <= 0 || D > 2147483647ll) return ASTRA_ERR_BAD_SHAPE;
+    if (T < 0 || Hh <= 0 || D <= 0 || D > 1073741823ll) return ASTRA_ERR_BAD_SHAPE;
     if (T > 0 && (Hh > kInt64Max / 4 / T || D > kInt64Max / 4 / (T * Hh))) return ASTRA_ERR_BAD_SHAPE;
+    if (T == 0) return ASTRA_OK;
+    if (!v_out || !v_a || !v_b || !lse_a || !lse_b) return ASTRA_ERR_NULL_POINTER;
     const int64_t U = units_per_elem(dtype);
     const size_t eb = static_cast<size_t>(2 * U);
     if (!aligned(v_out, eb) || !aligned(v_a, eb) || !aligned(v_b, eb) || !aligned(lse_a, 4) ||
         !aligned(lse_b, 4) || (lse_out && !aligned(lse_out, 4)))
         return ASTRA_ERR_MISALIGNED;
-    if (T == 0) return ASTRA_OK;
     const int64_t rows = T * Hh;
     const int64_t Du = D * U;  // row width in 16-bit units
     const int64_t vbytes = rows * Du * 2, sbytes = rows * 4;
@@ -506,18 +541,20 @@ astra_status_t astra_merge_attn_states_lse(void *v_out, float *lse_out, const vo
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     uint16_t *vo = static_cast<uint16_t *>(v_out);
     const uint16_t *va = static_cast<const uint16_t *>(v_a), *vb = static_cast<const uint16_t *>(v_b);
-    ASTRA_FOR_DTYPE(dtype, dispatch_merge<DT>(vo, lse_out, va, lse_a, vb, lse_b, rows, Du, stream));
-    return launch_status();
+    cudaError_t err = cudaSuccess;
+    ASTRA_FOR_DTYPE(dtype, err = dispatch_merge<DT>(vo, lse_out, va, lse_a, vb, lse_b, rows, Du, stream));
+    return launch_status(err);
 }
 
 astra_status_t astra_merge_attn_states_lse_ex(void *v_out, float *lse_out, const void *v_a,
                                               const float *lse_a, const void *v_b, const float *lse_b,
                                               int64_t T, int64_t Hh, int64_t D, const int64_t *strides,
                                               astra_dtype_t dtype, void *cuda_stream) {
-    if (!v_out || !v_a || !v_b || !lse_a || !lse_b || !strides) return ASTRA_ERR_NULL_POINTER;
     if (!valid_dtype(dtype)) return ASTRA_ERR_BAD_DTYPE;
-    if (T < 0 || Hh <= 0 || D <= 0 || D > 2147483647ll || Hh > 2147483647ll) return ASTRA_ERR_BAD_SHAPE;
-    if (T > 0 && T * Hh > 2147483647ll) return ASTRA_ERR_BAD_SHAPE;
+    if (T < 0 || Hh <= 0 || D <= 0 || D > 1073741823ll || Hh > 2147483647ll) return ASTRA_ERR_BAD_SHAPE;
+    if (T > 0 && Hh > 2147483647ll / T) return ASTRA_ERR_BAD_SHAPE;  // T * Hh must stay below 2^31
+    if (T == 0) return ASTRA_OK;
+    if (!v_out || !v_a || !v_b || !lse_a || !lse_b || !strides) return ASTRA_ERR_NULL_POINTER;
     for (int i = 0; i < 12; ++i) {
         if (lse_out == nullptr && i >= 10) break;
         // every offset (T-1)*stride, (Hh-1)*stride must stay far inside int64
@@ -536,7 +573,6 @@ astra_status_t astra_merge_attn_states_lse_ex(void *v_out, float *lse_out, const
     if (!aligned(v_out, eb) || !aligned(v_a, eb) || !aligned(v_b, eb) || !aligned(lse_a, 4) ||
         !aligned(lse_b, 4) || (lse_out && !aligned(lse_out, 4)))
         return ASTRA_ERR_MISALIGNED;
-    if (T == 0) return ASTRA_OK;
     // written tensors must have non-overlapping rows; read tensors may broadcast (stride 0)
     if (!rows_disjoint(T, Hh, Du, st.vo_t, st.vo_h)) return ASTRA_ERR_BAD_SHAPE;
     if (lse_out && !rows_disjoint(T, Hh, 1, st.so_t, st.so_h)) return ASTRA_ERR_BAD_SHAPE;
@@ -559,9 +595,12 @@ astra_status_t astra_merge_attn_states_lse_ex(void *v_out, float *lse_out, const
     uint16_t *vo = static_cast<uint16_t *>(v_out);
     const uint16_t *va = static_cast<const uint16_t *>(v_a), *vb = static_cast<const uint16_t *>(v_b);
     const int64_t rows = T * Hh;
-    ASTRA_FOR_DTYPE(dtype, dispatch_merge_strided<DT>(vo, lse_out, va, lse_a, vb, lse_b, rows, Hh, Du, st, stream));
-    return launch_status();
+    cudaError_t err = cudaSuccess;
+    ASTRA_FOR_DTYPE(dtype, err = dispatch_merge_strided<DT>(vo, lse_out, va, lse_a, vb, lse_b, rows, Hh, Du, st, stream));
+    return launch_status(err);
 }
+
+const char *astra_build_id(void) { return kBuildId + sizeof("astra-build-id:") - 1; }
 
 const char *astra_status_string(astra_status_t status) {
     switch (status) {

@@ -33,7 +33,7 @@ import torch  # noqa: E402
 
 import oracle  # noqa: E402
 from paper_2509_07506_b200 import workloads as wl  # noqa: E402
-from parity import check_lse, check_values  # noqa: E402
+from parity import check_lse, check_values, merge_floor  # noqa: E402
 
 
 def load(path: str) -> ctypes.CDLL:
@@ -90,7 +90,7 @@ def validate(lib) -> dict:
         assert st == 0, f"status {st}"
         ov, os_ = oracle.merge_attn_states_lse(wl.bits(inp.v_a), inp.lse_a.numpy(), wl.bits(inp.v_b),
                                                inp.lse_b.numpy(), dtype)
-        floor = 2.0 ** -22 * 2.0 * np.maximum(np.abs(_f64(inp.v_a)), np.abs(_f64(inp.v_b)))
+        floor = merge_floor(_f64(inp.v_a), inp.lse_a.numpy(), _f64(inp.v_b), inp.lse_b.numpy(), dtype)
         u = check_values(_f64(vo.cpu()), ov, dtype, extra=floor)["max_err_ulp"]
         check_lse(so.cpu().numpy(), os_)
         return u

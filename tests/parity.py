@@ -13,7 +13,9 @@ Gates (oracle values are fp64; GPU values are the exact values of its 16-bit out
     is rounded to binary32 before exp2, which costs |a| * 2^-24 relative: the gate there is
     (16 + 2*|a|) ulp, passed in through `extra`.
   - merge values: the blend a*Va + b*Vb can cancel, so the binary32 accumulation floor
-    2^-22 * (|a*Va| + |b*Vb|) is added to the gate.
+    2^-22 * (|a*Va| + |b*Vb|) is added to the gate (4 times that for fp32 storage, where the
+    weights' own few binary32 ulp are no longer hidden by the store's rounding).  `merge_floor` is
+    the one definition of that term; every merge comparison in the repository uses it.
   - merged score: |gpu - oracle| <= 1e-5; -inf must be -inf.
 """
 from __future__ import annotations
@@ -29,13 +31,29 @@ _GATE_ULPS = {BF16: 2.0, FP16: 2.0, FP32: 16.0}
 def ulp(v: np.ndarray, dtype: int) -> np.ndarray:
     """Spacing of the storage format at |v| (v != 0 finite); the subnormal quantum below the normals."""
     a = np.abs(np.asarray(v, dtype=np.float64))
-    with np.errstate(divide="ignore"):
-        e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
-    # guard against log2 rounding at exact powers of two
-    e = np.where(np.ldexp(1.0, e.astype(np.int64)) > a, e - 1, e)
-    e = np.where(np.ldexp(1.0, (e + 1).astype(np.int64)) <= a, e + 1, e)
-    e = np.maximum(e, _EMIN[dtype])
-    return np.ldexp(1.0, (e - _FRAC[dtype]).astype(np.int64))
+    _, e = np.frexp(a)                      # a = m * 2^e with m in [0.5, 1): floor(log2 a) = e - 1, exactly
+    e = np.maximum(e - 1, _EMIN[dtype])
+    return np.ldexp(1.0, e - _FRAC[dtype])
+
+
+def merge_floor(v_a, lse_a, v_b, lse_b, dtype: int) -> np.ndarray:
+    """binary32 accumulation floor of the two-term blend, 2^-22 * (|a*Va| + |b*Vb|) with (a, b) =
+    softmax([Sa, Sb]) in double precision (4 times that for fp32 storage).  v_*: [..., D] arrays of the
+    inputs' exact values, lse_*: [...] scores.  An empty side (-inf score) has weight 0 and its payload,
+    which may be Inf or NaN garbage, does not count; rows outside the domain (+inf or NaN scores) get 0."""
+    sa = np.asarray(lse_a, dtype=np.float64)[..., None]
+    sb = np.asarray(lse_b, dtype=np.float64)[..., None]
+    with np.errstate(invalid="ignore", over="ignore"):
+        m = np.maximum(sa, sb)
+        m = np.where(np.isfinite(m), m, 0.0)
+        ea, eb = np.exp(sa - m), np.exp(sb - m)
+        a, b = ea / (ea + eb), eb / (ea + eb)
+    a = np.nan_to_num(a, nan=0.0, posinf=0.0, neginf=0.0)
+    b = np.nan_to_num(b, nan=0.0, posinf=0.0, neginf=0.0)
+    va = np.nan_to_num(np.asarray(v_a, dtype=np.float64), nan=0.0, posinf=0.0, neginf=0.0)
+    vb = np.nan_to_num(np.asarray(v_b, dtype=np.float64), nan=0.0, posinf=0.0, neginf=0.0)
+    floor = 2.0 ** -22 * (np.abs(a * va) + np.abs(b * vb))
+    return 4.0 * floor if dtype == FP32 else floor
 
 
 def value_gate(oracle: np.ndarray, dtype: int, extra: np.ndarray | float = 0.0) -> np.ndarray:

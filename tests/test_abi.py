@@ -89,6 +89,42 @@ def test_rmsnorm_argument_errors(lib):
     assert f(A, A + 8, 3 * A, 1, 8, 1e-6, 0, None) == binding.ASTRA_ERR_OVERLAP
     assert f(A, 2 * A, A + 4, 1, 8, 1e-6, 0, None) == binding.ASTRA_ERR_OVERLAP
     assert f(A, 2 * A, 3 * A, 0, 8, 1e-6, 0, None) == binding.ASTRA_OK
+    # a row is indexed in 16-bit units with 32-bit integers: at most 2^30 units per row
+    assert f(A, 2 * A, 3 * A, 1, 2 ** 30 + 1, 1e-6, 0, None) == binding.ASTRA_ERR_BAD_SHAPE
+    assert f(A, 2 * A, 3 * A, 1, 2 ** 29 + 1, 1e-6, binding.ASTRA_FP32, None) == binding.ASTRA_ERR_BAD_SHAPE
+    assert f(A, 2 * A, 3 * A, 0, 2 ** 30, 1e-6, 0, None) == binding.ASTRA_OK
+    assert f(A, 2 * A, 3 * A, 0, 2 ** 29, 1e-6, binding.ASTRA_FP32, None) == binding.ASTRA_OK
+
+
+def test_empty_batches_do_not_examine_their_pointers(lib):
+    """T == 0: an empty tensor may have a NULL address (torch reports 0 for it), the call is ASTRA_OK;
+    shape and dtype errors are still reported."""
+    assert lib.astra_fused_add_rmsnorm(None, None, None, 0, 8, 1e-6, 0, None) == binding.ASTRA_OK
+    assert lib.astra_fused_add_rmsnorm_ex(None, None, None, None, None, 0, 8, 8, 8, 8, 8, 1e-6, 1, None) == binding.ASTRA_OK
+    assert lib.astra_silu_and_mul(None, None, 0, 8, 0, None) == binding.ASTRA_OK
+    assert lib.astra_silu_and_mul_ex(None, None, None, 0, 8, 8, 8, 8, 2, None) == binding.ASTRA_OK
+    assert lib.astra_merge_attn_states_lse(None, None, None, None, None, None, 0, 2, 8, 0, None) == binding.ASTRA_OK
+    assert lib.astra_merge_attn_states_lse_ex(None, None, None, None, None, None, 0, 2, 8, None, 0, None) == binding.ASTRA_OK
+    assert lib.astra_fused_add_rmsnorm(None, None, None, 0, 0, 1e-6, 0, None) == binding.ASTRA_ERR_BAD_SHAPE
+    assert lib.astra_silu_and_mul(None, None, 0, 8, 9, None) == binding.ASTRA_ERR_BAD_DTYPE
+    assert lib.astra_merge_attn_states_lse(None, None, None, None, None, None, 0, 0, 8, 0, None) == binding.ASTRA_ERR_BAD_SHAPE
+
+
+def test_refused_launch_is_reported_and_stops_the_call(lib):
+    """Where no CUDA device exists the runtime refuses every launch on the host: a well-formed call
+    must come back as ASTRA_ERR_CUDA (the launch's own status), again on the next call (nothing is
+    left pending in between), and argument errors keep their own codes.  Skipped where a device
+    exists: the fake addresses below must never reach a GPU."""
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a CUDA device is present; the fake addresses of this test must not be launched on")
+    for _ in range(2):
+        assert lib.astra_fused_add_rmsnorm(A, 2 * A, 3 * A, 4, 4096, 1e-6, 0, None) == binding.ASTRA_ERR_CUDA
+        assert lib.astra_fused_add_rmsnorm(A, 16 * A, 32 * A, 2, 40000, 1e-6, 0, None) == binding.ASTRA_ERR_CUDA  # cluster launch
+        assert lib.astra_silu_and_mul(A, 16 * A, 4, 1024, 1, None) == binding.ASTRA_ERR_CUDA
+        assert lib.astra_merge_attn_states_lse(A, 2 * A, 3 * A, 4 * A, 5 * A, 6 * A, 4, 2, 128, 0, None) == binding.ASTRA_ERR_CUDA
+        assert lib.astra_silu_and_mul(A, None, 4, 1024, 1, None) == binding.ASTRA_ERR_NULL_POINTER
+    assert "launch" in lib.astra_status_string(binding.ASTRA_ERR_CUDA).decode()
 
 
 def test_silu_argument_errors(lib):
@@ -187,6 +223,8 @@ def test_merge_ex_argument_errors(lib):
     assert call(v_b=None) == binding.ASTRA_ERR_NULL_POINTER
     assert call(dtype=3) == binding.ASTRA_ERR_BAD_DTYPE
     assert call(T=2 ** 31, Hh=2) == binding.ASTRA_ERR_BAD_SHAPE
+    assert call(T=2 ** 62, Hh=4) == binding.ASTRA_ERR_BAD_SHAPE   # T * Hh would wrap a 64-bit product
+    assert call(T=2 ** 33, Hh=2 ** 31 - 1) == binding.ASTRA_ERR_BAD_SHAPE
     neg = list(dense); neg[0] = -16
     assert call(strides=neg) == binding.ASTRA_ERR_BAD_SHAPE
     squeezed = list(dense); squeezed[5] = 4           # v_out head stride < D: rows overlap

@@ -8,7 +8,7 @@ import torch
 import oracle
 from paper_2509_07506_b200 import ablation
 from paper_2509_07506_b200 import workloads as wl
-from parity import check_lse, check_values
+from parity import check_lse, check_values, merge_floor
 
 pytestmark = pytest.mark.gpu
 BF16, FP16 = wl.BF16, wl.FP16
@@ -51,6 +51,6 @@ def test_ablation_merge(design, dtype, T, Hh, D):
     vo, so = torch.zeros_like(va), torch.zeros_like(sa)
     ablation.astra_ablation_merge_attn_states_lse(design, vo, so, va, sa, vb, sb)
     ov, os_ = oracle.merge_attn_states_lse(wl.bits(inp.v_a), inp.lse_a.numpy(), wl.bits(inp.v_b), inp.lse_b.numpy(), dtype)
-    floor = 2.0 ** -22 * 2.0 * np.maximum(np.abs(f64(inp.v_a)), np.abs(f64(inp.v_b)))
+    floor = merge_floor(f64(inp.v_a), inp.lse_a.numpy(), f64(inp.v_b), inp.lse_b.numpy(), dtype)
     check_values(f64(vo.cpu()), ov, dtype, extra=floor, what=f"ablation merge design {design}")
     check_lse(so.cpu().numpy(), os_, what=f"ablation merge design {design}")

@@ -8,7 +8,7 @@ import torch
 import oracle
 import paper_2509_07506_b200 as astra
 from paper_2509_07506_b200 import workloads as wl
-from parity import check_lse, check_values
+from parity import check_lse, check_values, merge_floor
 from test_gpu_parity import run_merge, run_rmsnorm, run_silu
 
 pytestmark = pytest.mark.gpu
@@ -60,6 +60,6 @@ def test_fp32_pitched_and_out_of_place():
     vo = torch.zeros_like(va); so = torch.zeros((4, 19), device="cuda").t()
     astra.astra_merge_attn_states_lse_ex(vo, so, va, sa, vb, sb)
     ov, os_ = oracle.merge_attn_states_lse(wl.bits(mi.v_a), mi.lse_a.numpy(), wl.bits(mi.v_b), mi.lse_b.numpy(), FP32)
-    floor = 2.0 ** -20 * 2.0 * np.maximum(np.abs(mi.v_a.double().numpy()), np.abs(mi.v_b.double().numpy()))
+    floor = merge_floor(mi.v_a.double().numpy(), mi.lse_a.numpy(), mi.v_b.double().numpy(), mi.lse_b.numpy(), FP32)
     check_values(vo.cpu().double().numpy(), ov, FP32, extra=floor, what="merge_ex fp32")
     check_lse(so.cpu().numpy(), os_, what="merge_ex fp32")

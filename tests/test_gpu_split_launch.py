@@ -10,7 +10,7 @@ import torch
 import oracle
 from paper_2509_07506_b200 import build as astra_build
 from paper_2509_07506_b200 import workloads as wl
-from parity import check_lse, check_values
+from parity import check_lse, check_values, merge_floor
 
 pytestmark = pytest.mark.gpu
 BF16 = wl.BF16
@@ -70,6 +70,6 @@ def test_merge_rows_split_over_launches(small_limits_lib, strided):
                                                           vb.data_ptr(), sb.data_ptr(), T, Hh, D, 0, None)
     assert st == 0
     ov, os_ = oracle.merge_attn_states_lse(wl.bits(inp.v_a), inp.lse_a.numpy(), wl.bits(inp.v_b), inp.lse_b.numpy(), BF16)
-    floor = 2.0 ** -22 * 2.0 * np.maximum(np.abs(f64(inp.v_a)), np.abs(f64(inp.v_b)))
+    floor = merge_floor(f64(inp.v_a), inp.lse_a.numpy(), f64(inp.v_b), inp.lse_b.numpy(), BF16)
     check_values(f64(vo.cpu()), ov, BF16, extra=floor, what="merge split")
     check_lse(so.cpu().numpy(), os_, what="merge split")

@@ -9,7 +9,7 @@ import torch
 import oracle
 import paper_2509_07506_b200 as astra
 from paper_2509_07506_b200 import workloads as wl
-from parity import check_lse, check_values
+from parity import check_lse, check_values, merge_floor
 
 pytestmark = pytest.mark.gpu
 
@@ -133,7 +133,7 @@ def test_merge_ex_strided(dtype, Hh, D, layout):
     astra.astra_merge_attn_states_lse_ex(vo, so, va, sa, vb, sb)
     torch.cuda.synchronize()
     ov, os_ = oracle.merge_attn_states_lse(wl.bits(inp.v_a), inp.lse_a.numpy(), wl.bits(inp.v_b), inp.lse_b.numpy(), dtype)
-    floor = 2.0 ** -22 * 2.0 * np.maximum(np.abs(f64(inp.v_a)), np.abs(f64(inp.v_b)))
+    floor = merge_floor(f64(inp.v_a), inp.lse_a.numpy(), f64(inp.v_b), inp.lse_b.numpy(), dtype)
     check_values(f64(vo.cpu()), ov, dtype, extra=floor, what="merge_ex")
     check_lse(so.cpu().numpy(), os_, what="merge_ex lse")
     for buf in bufs:
