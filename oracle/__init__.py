@@ -78,6 +78,9 @@ def declare(lib):
     lib.oracle_fused_add_rmsnorm.argtypes = [u16p, u16p, u16p, i64, i64, ctypes.c_float,
                                              ctypes.c_int, f64p, u16p, ctypes.c_int]
     lib.oracle_fused_add_rmsnorm.restype = None
+    lib.oracle_fused_allreduce_add_rmsnorm.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.c_int, u16p, u16p, i64,
+                                                       i64, ctypes.c_float, ctypes.c_int, f64p, u16p, ctypes.c_int]
+    lib.oracle_fused_allreduce_add_rmsnorm.restype = None
     lib.oracle_silu_and_mul.argtypes = [u16p, i64, i64, ctypes.c_int, f64p, ctypes.c_int]
     lib.oracle_silu_and_mul.restype = None
     lib.oracle_merge_attn_states_lse.argtypes = [u16p, f32p, u16p, f32p, i64, i64, i64,
@@ -140,6 +143,27 @@ def fused_add_rmsnorm(x, residual, weight, eps: float, dtype: int, nthreads: int
     r_out = np.empty((T, H), dtype=x.dtype)
     _load().oracle_fused_add_rmsnorm(
         _ptr(x, ctypes.c_uint16), _ptr(residual, ctypes.c_uint16), _ptr(weight, ctypes.c_uint16),
+        T, H, np.float32(eps).item(), int(dtype),
+        _ptr(y, ctypes.c_double), _ptr(r_out, ctypes.c_uint16), int(nthreads))
+    return y, r_out
+
+
+def fused_allreduce_add_rmsnorm(parts, residual, weight, eps: float, dtype: int, nthreads: int = 1):
+    """Kernel 2 of Table 1 on a hidden state given as N partial sums ``parts`` (a sequence of [T, H]
+    pattern arrays in rank order): binary32 additions in rank order, the residual last.
+    Returns (y float64 [T,H], residual_out storage patterns [T,H])."""
+    if len(parts) < 1:
+        raise ValueError("at least one partial is needed")
+    first = np.ascontiguousarray(parts[0])
+    T, H = first.shape
+    parts = [_u16(p, (T, H), dtype) for p in parts]
+    residual = _u16(residual, (T, H), dtype)
+    weight = _u16(weight, (H,), dtype)
+    table = (ctypes.c_void_p * len(parts))(*[p.ctypes.data for p in parts])
+    y = np.empty((T, H), dtype=np.float64)
+    r_out = np.empty((T, H), dtype=first.dtype)
+    _load().oracle_fused_allreduce_add_rmsnorm(
+        table, len(parts), _ptr(residual, ctypes.c_uint16), _ptr(weight, ctypes.c_uint16),
         T, H, np.float32(eps).item(), int(dtype),
         _ptr(y, ctypes.c_double), _ptr(r_out, ctypes.c_uint16), int(nthreads))
     return y, r_out

@@ -25,7 +25,10 @@
  * (plain RMSNorm, two-way softmax, attention over a split key set), library
  * routines of torch on CPU in fp64, an integer-only bf16 adder for the
  * residual sum, and torch's own float->bf16 / float->fp16 casts for the
- * rounding helpers.  No function here is "parity unpinned".
+ * rounding helpers; for the partial-sum form of Kernel 2 an exact-rational
+ * adder with its own binary32 rounding, cases whose result depends on the
+ * order and on the number of roundings, and its N = 1 case against
+ * fused_add_rmsnorm.  No function here is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -196,6 +199,69 @@ void oracle_fused_add_rmsnorm(const void *x, const void *r, const void *w,
         for (int64_t j = 0; j < H; ++j) {
             double xv = load_value(x, t * H + j, dtype, f), rv = load_value(r, t * H + j, dtype, f);
             float s32 = add_binary32(xv, rv, dtype);
+            store_rounded(residual_out, t * H + j, s32, dtype, f);
+            y_out[t * H + j] = (double)s32 / denom * load_value(w, j, dtype, f);
+        }
+    }
+}
+
+/*
+ * fused_allreduce_add_rmsnorm: Kernel 2 of Table 1 applied to a hidden state that arrives as N
+ * partial sums, one per tensor-parallel rank (the all-reduce that precedes the operation in
+ * tensor-parallel serving, folded into it):
+ *     x = x_0 + x_1 + ... + x_{N-1};   s = x + r;   r_out <- s;   y = s / sqrt(mean(s^2) + eps) (.) w
+ *
+ * parts : N pointers to [T, H] storage patterns, in rank order.  r : [T, H].  w : [H].
+ * y_out : [T, H] doubles.  residual_out : [T, H] storage patterns.
+ *
+ * Readings (the paper states Kernel 2 for one x only; where the additions are rounded has to be
+ * fixed because the updated residual is compared bit for bit):
+ *  - every addition is one binary32 addition (round to nearest even): the partials are added in
+ *    rank order starting from x_0, then the residual is added last:
+ *        s = fl( fl( ... fl( fl(x_0 + x_1) + x_2 ) ... + x_{N-1} ) + r ).
+ *    N = 1 is fused_add_rmsnorm exactly.  Rank order makes every rank of a tensor-parallel group
+ *    compute the same bits.
+ *  - nothing is rounded to the storage type before the residual joins (a separate all-reduce
+ *    would have rounded x there); the residual gets s rounded once to the storage type;
+ *  - the norm uses the binary32 s; eps and the weight as in fused_add_rmsnorm.
+ * The C type float is binary32 and this file is compiled without contraction or excess precision,
+ * so `a + b` on floats is that one addition; the volatile keeps the compiler from re-associating.
+ */
+static float value_as_float(const void *base, int64_t i, int dtype, storage_format f)
+{
+    /* every storage pattern is exactly representable in binary32 */
+    return (float)load_value(base, i, dtype, f);
+}
+
+static float sum_in_rank_order(const void *const *parts, int n_parts, const void *r, int64_t i,
+                               int dtype, storage_format f)
+{
+    volatile float acc = value_as_float(parts[0], i, dtype, f);
+    for (int p = 1; p < n_parts; ++p) {
+        volatile float next = value_as_float(parts[p], i, dtype, f);
+        acc = acc + next;
+    }
+    volatile float res = value_as_float(r, i, dtype, f);
+    acc = acc + res;
+    return acc;
+}
+
+void oracle_fused_allreduce_add_rmsnorm(const void *const *parts, int n_parts, const void *r,
+                                        const void *w, int64_t T, int64_t H, float eps, int dtype,
+                                        double *y_out, void *residual_out, int nthreads)
+{
+    storage_format f = format_of(dtype);
+    if (nthreads < 1) nthreads = 1;
+#pragma omp parallel for num_threads(nthreads) schedule(static)
+    for (int64_t t = 0; t < T; ++t) {
+        double sum_sq = 0.0;
+        for (int64_t j = 0; j < H; ++j) {
+            double s = (double)sum_in_rank_order(parts, n_parts, r, t * H + j, dtype, f);
+            sum_sq += s * s;
+        }
+        double denom = sqrt(sum_sq / (double)H + (double)eps);
+        for (int64_t j = 0; j < H; ++j) {
+            float s32 = sum_in_rank_order(parts, n_parts, r, t * H + j, dtype, f);
             store_rounded(residual_out, t * H + j, s32, dtype, f);
             y_out[t * H + j] = (double)s32 / denom * load_value(w, j, dtype, f);
         }

@@ -34,6 +34,33 @@ MUTATIONS = [
      "float s32 = add_binary32(xv, rv, dtype);", "float s32 = (float)xv;"),
     ("rmsnorm: divides by the mean square instead of its root",
      "double denom = sqrt(", "double denom = ("),
+    ("allreduce form: the residual is not added",
+     "    acc = acc + res;\n", "    acc = acc + 0.0f * res;\n"),
+    ("allreduce form: the last partial is skipped",
+     "for (int p = 1; p < n_parts; ++p) {", "for (int p = 1; p < n_parts - 1; ++p) {"),
+    ("allreduce form: partials added from the last rank down",
+     "volatile float acc = value_as_float(parts[0], i, dtype, f);\n    for (int p = 1; p < n_parts; ++p) {\n"
+     "        volatile float next = value_as_float(parts[p], i, dtype, f);",
+     "volatile float acc = value_as_float(parts[n_parts - 1], i, dtype, f);\n    for (int p = 1; p < n_parts; ++p) {\n"
+     "        volatile float next = value_as_float(parts[n_parts - 1 - p], i, dtype, f);"),
+    ("allreduce form: the residual is added first",
+     "volatile float acc = value_as_float(parts[0], i, dtype, f);\n    for (int p = 1; p < n_parts; ++p) {\n"
+     "        volatile float next = value_as_float(parts[p], i, dtype, f);",
+     "volatile float acc = value_as_float(r, i, dtype, f) + value_as_float(parts[0], i, dtype, f);\n"
+     "    r = parts[0];\n    for (int p = 1; p <= n_parts; ++p) {\n"
+     "        volatile float next = p < n_parts ? value_as_float(parts[p], i, dtype, f) : 0.0f;"),
+    ("allreduce form: the sum is carried in double and rounded once",
+     "volatile float acc = value_as_float(parts[0], i, dtype, f);", "volatile double acc = value_as_float(parts[0], i, dtype, f);"),
+    ("allreduce form: the summed state is rounded to the storage type before the residual joins",
+     "    volatile float res = value_as_float(r, i, dtype, f);",
+     "    if (dtype != ORACLE_FP32) acc = (float)widen(round_to_storage((double)acc, f), f);\n"
+     "    volatile float res = value_as_float(r, i, dtype, f);"),
+    ("allreduce form: norm taken from the stored residual",
+     "double s = (double)sum_in_rank_order(parts, n_parts, r, t * H + j, dtype, f);",
+     "double s = dtype == ORACLE_FP32 ? 0.0 : widen(round_to_storage((double)sum_in_rank_order(parts, n_parts, r, t * H + j, dtype, f), f), f);"),
+    ("allreduce form: every element reads the first row of the partials",
+     "(double)sum_in_rank_order(parts, n_parts, r, t * H + j, dtype, f);\n            sum_sq",
+     "(double)sum_in_rank_order(parts, n_parts, r, j, dtype, f);\n            sum_sq"),
     ("silu: e^{+z} in the denominator",
      "return z / (1.0 + exp(-z));", "return z / (1.0 + exp(z));"),
     ("silu: sigmoid instead of SiLU (z dropped)",

@@ -297,6 +297,139 @@ def test_rmsnorm_rows_are_independent_and_weight_indexed_by_column():
 
 
 # ---------------------------------------------------------------------------------------
+# fused_allreduce_add_rmsnorm: Kernel 2 on a hidden state given as N partial sums
+# ---------------------------------------------------------------------------------------
+
+def _fl32(q):
+    """Correctly rounded (nearest-even) binary32 value of an exact rational, as an exact rational:
+    integer arithmetic only.  Magnitudes stay inside the normal range of binary32 in these tests."""
+    from fractions import Fraction
+    if q == 0:
+        return Fraction(0)
+    sign, a = (-1 if q < 0 else 1), abs(q)
+    e = a.numerator.bit_length() - a.denominator.bit_length()
+    if Fraction(2) ** e > a:
+        e -= 1                                    # now 2^e <= a < 2^(e+1)
+    assert -126 <= e <= 127
+    quantum = Fraction(2) ** (e - 23)
+    n, rem = divmod(a, quantum)                    # a = n * quantum + rem, n a 24-bit integer
+    if rem * 2 > quantum or (rem * 2 == quantum and n % 2 == 1):
+        n += 1
+    return sign * n * quantum
+
+
+def _rank_order_sum(values, r):
+    """fl(...fl(fl(x0 + x1) + x2)... + r) with exact rationals and _fl32."""
+    acc = values[0]
+    for v in values[1:]:
+        acc = _fl32(acc + v)
+    return _fl32(acc + r)
+
+
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
+@pytest.mark.parametrize("n_parts", [1, 2, 3, 5, 8])
+def test_allreduce_form_against_exact_rational_adder(dtype, n_parts):
+    """Every element: the rank-order binary32 sum rebuilt from exact rationals with an integer-only
+    rounding; the residual is that sum cast once by torch; y follows from the sums in fp64.  The inputs
+    span many binades, so most additions are inexact and both their order and their number matter."""
+    from fractions import Fraction
+    T, H = 3, 29
+    g = torch.Generator().manual_seed(100 + n_parts)
+    span = 6 if dtype == FP16 else 12
+
+    def draw(shape):
+        mant = 1 + torch.rand(shape, generator=g, dtype=torch.float64)
+        expo = torch.randint(-span, span + 1, shape, generator=g)
+        sign = torch.randint(0, 2, shape, generator=g) * 2 - 1
+        return (sign * mant * 2.0 ** expo).to(TD[dtype])
+
+    parts = [draw((T, H)) for _ in range(n_parts)]
+    r, w = draw((T, H)), draw((H,))
+    eps = 1e-5
+    y, r_out = oracle.fused_allreduce_add_rmsnorm([wl.bits(p) for p in parts], wl.bits(r), wl.bits(w), eps, dtype)
+    s = np.empty((T, H))
+    for t in range(T):
+        for j in range(H):
+            q = _rank_order_sum([Fraction(float(p[t, j])) for p in parts], Fraction(float(r[t, j])))
+            s[t, j] = float(q)                     # a binary32 value: exact in a double
+    assert np.array_equal(r_out, wl.bits(torch.from_numpy(s).to(torch.float32).to(TD[dtype])))
+    denom = np.sqrt((s * s).mean(axis=1, keepdims=True) + float(np.float32(eps)))
+    np.testing.assert_allclose(y, s / denom * w.to(torch.float64).numpy(), rtol=1e-13)
+
+
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
+def test_allreduce_form_with_one_partial_is_fused_add_rmsnorm(dtype):
+    inp = wl.rmsnorm_inputs(9, 133, dtype, eps=1e-5, seed=31)
+    xb, rb, wb = wl.bits(inp.x), wl.bits(inp.residual), wl.bits(inp.weight)
+    y1, r1 = oracle.fused_allreduce_add_rmsnorm([xb], rb, wb, 1e-5, dtype)
+    y0, r0 = oracle.fused_add_rmsnorm(xb, rb, wb, 1e-5, dtype)
+    assert np.array_equal(y1, y0) and np.array_equal(r1, r0)
+
+
+@pytest.mark.parametrize("dtype", VALUE_DTYPES)
+def test_allreduce_form_equals_kernel_2_on_the_summed_state_when_the_sums_are_exact(dtype):
+    """Small integers: every partial sum is exact and fits the storage type, so the N-partial form is
+    Kernel 2 applied to x = sum of the partials, in any order of the partials."""
+    g = torch.Generator().manual_seed(5)
+    parts = [torch.randint(-7, 8, (4, 40), generator=g).to(TD[dtype]) for _ in range(6)]
+    r = torch.randint(-7, 8, (4, 40), generator=g).to(TD[dtype])
+    w = (1 + 0.1 * torch.randn(40, generator=g)).to(TD[dtype])
+    x = sum(p.to(torch.float64) for p in parts).to(TD[dtype])
+    y0, r0 = oracle.fused_add_rmsnorm(wl.bits(x), wl.bits(r), wl.bits(w), 1e-6, dtype)
+    for order in ([0, 1, 2, 3, 4, 5], [5, 3, 1, 0, 2, 4]):
+        y, ro = oracle.fused_allreduce_add_rmsnorm([wl.bits(parts[i]) for i in order], wl.bits(r), wl.bits(w), 1e-6, dtype)
+        assert np.array_equal(ro, r0)
+        np.testing.assert_allclose(y, y0, rtol=1e-15)
+
+
+def test_allreduce_form_order_and_roundings():
+    """Hand cases whose answer depends on the reading: rank order, the residual last, one rounding
+    per addition (not one for the whole sum), and no rounding to the storage type before the residual."""
+    def run(parts, r, dtype):
+        y, ro = oracle.fused_allreduce_add_rmsnorm([enc([[v]], dtype) for v in parts], enc([[r]], dtype),
+                                                   enc([1.0], dtype), 1e-6, dtype)
+        return y[0, 0], ro
+    big, tiny = 256.0, 2.0 ** -17          # tiny is a quarter of a binary32 ulp of big
+    # rank order: (big - big) + tiny = tiny, but (big + tiny) - big = 0
+    y, ro = run([big, -big, tiny], 0.0, BF16)
+    assert np.array_equal(ro, enc([[tiny]], BF16)) and y > 0.0
+    y, ro = run([big, tiny, -big], 0.0, BF16)
+    assert np.array_equal(ro, enc([[0.0]], BF16)) and y == 0.0
+    # the residual joins last: (big + tiny) + (-big) = 0, whereas (-big + big) + tiny would be tiny
+    _, ro = run([big, tiny], -big, BF16)
+    assert np.array_equal(ro, enc([[0.0]], BF16))
+    _, ro = run([-big, tiny], big, BF16)
+    assert np.array_equal(ro, enc([[0.0]], BF16))
+    # one rounding per addition: 1 + 2^-24 + 2^-24 stays 1 step by step (ties to even twice);
+    # a sum carried in wider precision and rounded once would give 1 + 2^-23
+    _, ro = run([1.0, 2.0 ** -24, 2.0 ** -24], 0.0, FP32)
+    assert np.array_equal(ro, enc([[1.0]], FP32))
+    _, ro = run([2.0 ** -24, 2.0 ** -24, 1.0], 0.0, FP32)
+    assert np.array_equal(ro, enc([[1.0 + 2.0 ** -23]], FP32))
+    # nothing is rounded to the storage type before the residual joins: 1 + 2^-9 is not a bf16 value
+    _, ro = run([1.0, 2.0 ** -9], -1.0, BF16)
+    assert np.array_equal(ro, enc([[2.0 ** -9]], BF16))
+
+
+def test_allreduce_form_norm_uses_the_binary32_sum_and_constant_rows():
+    s0 = 1.0 + 2.0 ** -9
+    parts = [enc([[0.5, 0.25]], BF16), enc([[0.5, 0.25]], BF16), enc([[2.0 ** -9, 0.25]], BF16)]
+    y, ro = oracle.fused_allreduce_add_rmsnorm(parts, enc([[0.0, 0.25]], BF16), enc([1.0, 1.0], BF16), 0.0, BF16)
+    assert np.array_equal(ro, enc([[1.0, 1.0]], BF16))
+    assert y[0, 0] == pytest.approx(s0 / math.sqrt((s0 * s0 + 1.0) / 2.0), rel=1e-15)
+    assert y[0, 1] == pytest.approx(1.0 / math.sqrt((s0 * s0 + 1.0) / 2.0), rel=1e-15)
+    # constant row: every partial and the residual constant -> y = sign(c) * w / sqrt(1 + eps / c^2)
+    H, eps = 19, 1e-6
+    wt = torch.linspace(0.5, 1.5, H, dtype=torch.float64).to(torch.float16)
+    for c_parts, c_r in (([0.5, 0.25, 1.0], 0.25), ([-1.0, -0.5], -0.5)):
+        c = sum(c_parts) + c_r
+        y, _ = oracle.fused_allreduce_add_rmsnorm([enc([[v] * H], FP16) for v in c_parts], enc([[c_r] * H], FP16),
+                                                  wl.bits(wt), eps, FP16)
+        want = c / math.sqrt(c * c + float(np.float32(eps))) * wt.to(torch.float64).numpy()
+        np.testing.assert_allclose(y[0], want, rtol=1e-14)
+
+
+# ---------------------------------------------------------------------------------------
 # silu_and_mul  (Table 1, Kernel 3)
 # ---------------------------------------------------------------------------------------
 
@@ -522,6 +655,15 @@ def test_tiny_shapes_against_50_digit_arithmetic(dtype):
                         for d in range(Dm):
                             want = (ea * _D(a64[t, h, d]) + eb * _D(b64[t, h, d])) / (ea + eb)
                             assert float(want) == pytest.approx(v[t, h, d], rel=1e-13, abs=1e-15)
+
+
+def test_threads_do_not_change_the_allreduce_form():
+    g = torch.Generator().manual_seed(8)
+    parts = [wl.bits(torch.randn((37, 65), generator=g).to(torch.bfloat16)) for _ in range(4)]
+    inp = wl.rmsnorm_inputs(37, 65, BF16, seed=2)
+    a = oracle.fused_allreduce_add_rmsnorm(parts, wl.bits(inp.residual), wl.bits(inp.weight), 1e-5, BF16, nthreads=1)
+    b = oracle.fused_allreduce_add_rmsnorm(parts, wl.bits(inp.residual), wl.bits(inp.weight), 1e-5, BF16, nthreads=4)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
 
 
 def test_threads_do_not_change_results():
