@@ -10,7 +10,7 @@ fraction is taken against the measured copy bandwidth of the GPU.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl astra|reference] [--no-sweep]
 
-N > 1 (under torchrun): every rank runs its own T = 8192 batch (weak scaling; the operations are
+N > 1 (under torchrun, or started plainly, in which case the N ranks are spawned here): every rank runs its own T = 8192 batch (weak scaling; the operations are
 independent per row, so there is no collective on the data path); time is the max over ranks.
 `--impl reference` times the fp64 CPU oracle on the host cores instead (rank 0 only).
 Exactly one JSON line is printed on stdout by rank 0.
@@ -37,18 +37,33 @@ from paper_2509_07506_b200 import workloads as wl  # noqa: E402
 
 METRIC = "achieved_hbm_bandwidth_llama3_8b_prefill_chain"
 UNIT = "GB/s"
-NOMINAL_HBM_GBS = 7700.0
+NOMINAL_HBM_GBS = 7700.0   # HGX B200 data-sheet figure
+HBM3E_SPEC_GBS = 8000.0    # 3996 MHz x 2 x 8192 bit: the interface's own ceiling
 FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 * 1024 * 1024
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_traffic_T4096.json")
 
-# Per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) at T = 8192 from the ncu
-# capture summarised in profiles/chain_T8192_launch_list.md.  An entry is removed (reported as null)
-# whenever its kernel changes after the capture.
-NCU_TRAFFIC_BYTES_T8192 = {
-    "silu_and_mul": 669.8e6,
-    "fused_add_rmsnorm": 208.7e6,
-    "merge_attn_states_lse": 164.0e6,
-}
+
+def ncu_traffic(kernel: str, tokens: int):
+    """Per-launch memory traffic of `kernel` at `tokens` rows from the profiler counters kept beside
+    the profile summaries: DRAM bytes read plus the bytes the SMs wrote into L2 (all of which reach
+    DRAM, a part of them only after the launch has ended, which is why the DRAM write counter of a
+    single profiled launch falls short).  The capture was taken at a smaller row count; traffic is
+    proportional to rows.  None when the counters are missing (for instance after a kernel changed)."""
+    try:
+        with open(TRAFFIC_FILE) as fh:
+            rec = json.load(fh)
+        k = rec["kernels"][kernel]
+        return round((k["dram_read_bytes"] + k["l2_write_bytes_from_sm"]) * tokens / rec["tokens"])
+    except Exception:
+        return None
+
+
+def fractions(gbs: float, peak: float) -> dict:
+    """A bandwidth against the three denominators in use: the copy bandwidth measured on this machine
+    (the roofline the benchmark reports against), the data-sheet figure and the interface ceiling."""
+    return {"frac_of_measured_peak": round(gbs / peak, 4), "frac_of_nominal_7700": round(gbs / NOMINAL_HBM_GBS, 4),
+            "frac_of_hbm3e_spec_8000": round(gbs / HBM3E_SPEC_GBS, 4)}
 
 
 def chain_bytes(T: int) -> dict:
@@ -160,7 +175,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
     torch.cuda.set_device(dev)
     from paper_2509_07506_b200 import build as astra_build
     if rank == 0:
-        astra_build.ensure_built()  # no-op when the library is newer than its sources; a missing library is fatal
+        astra_build.ensure_built()  # no-op when the library matches its sources; a missing or stale library is rebuilt or fatal
     if world > 1:
         dist.barrier()
     astra.load_library()  # fails loudly if the CUDA library is missing
@@ -295,8 +310,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
     for n in names:
         gbs = nbytes[n] / (kernel_ms[n] * 1e-3) / 1e9
         per_kernel[n] = {"us_per_call": round(kernel_ms[n] * 1e3, 2), "algorithmic_bytes": nbytes[n],
-                         "gbs": round(gbs, 1), "frac_of_measured_peak": round(gbs / peak, 4),
-                         "frac_of_nominal_7700": round(gbs / NOMINAL_HBM_GBS, 4)}
+                         "gbs": round(gbs, 1), **fractions(gbs, peak), "ncu_traffic_bytes": ncu_traffic(n, T)}
     dominant = max(names, key=lambda n: kernel_ms[n])
     dom_gbs = nbytes[dominant] / (kernel_ms[dominant] * 1e-3) / 1e9
     result = {
@@ -304,9 +318,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
         "ms_per_step": round(total_ms / K, 5), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "storage_dtype": "bf16", "data": "synthetic",
         "config": {
-            "workload": f"configs[4]: Llama-3-8B prefill-shaped chain, T={T} per GPU, bf16: "
-                        f"fused_add_rmsnorm [{T},4096] -> silu_and_mul [{T},2*14336] -> "
-                        f"merge_attn_states_lse [{T},32,128]",
+            "workload": chain_workload_name(T),
             "tokens_per_gpu": T, "seed": 4,
             "l2_policy": "inputs larger than L2: each step touches %.0f MB (L2 is 126 MB) and every kernel's "
                          "own working set exceeds L2, so nothing is re-used across launches" % (step_bytes / 1e6),
@@ -315,14 +327,19 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
         "per_kernel": per_kernel,
         "per_kernel_how": f"each kernel alone: {K} back-to-back launches between two CUDA events, after the chain region",
         "roofline": {"bound": "hbm", "kernel": dominant, "achieved": round(dom_gbs, 1), "peak": peak,
-                     "unit": "GB/s", "frac": round(dom_gbs / peak, 4), "traffic": NCU_TRAFFIC_BYTES_T8192.get(dominant) if T == wl.CHAIN_T else None,
-                     "peak_source": peak_source, "algorithmic_bytes_per_launch": nbytes[dominant]},
+                     "unit": "GB/s", "frac": round(dom_gbs / peak, 4), "traffic": ncu_traffic(dominant, T),
+                     "traffic_how": "ncu, per launch: dram__bytes_read.sum + bytes written into L2 by the SMs "
+                                    "(lts__t_sectors_srcunit_tex_op_write.sum x 32), captured at T=4096 and scaled by rows",
+                     "peak_source": peak_source, "algorithmic_bytes_per_launch": nbytes[dominant],
+                     "frac_of_hbm3e_spec_8000": round(dom_gbs / HBM3E_SPEC_GBS, 4),
+                     "frac_of_nominal_7700": round(dom_gbs / NOMINAL_HBM_GBS, 4)},
         "e2e": {"value": round(world * step_bytes * Ke / (e2e_ms * 1e-3) / 1e9, 2), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": Ke,
                 "ms_per_step": round(e2e_ms / Ke, 3),
                 "how": f"pinned host -> device, kernels, device -> pinned host for every tensor of every step, in "
                        f"{chunk}-row chunks pipelined over three streams (upload / compute / download)"},
         "gpu_launches": 6 * K + 3 * Ke * (-(-T // chunk)),  # chain + per-kernel regions + chunked end-to-end steps
+        "launcher": os.environ.get("ASTRA_BENCH_LAUNCHER", "external launcher" if world > 1 else "single process"),
         "clocks": sampler.summary([(t_wall0, t_wall1), (t_wall2, t_wall3)]) if sampler else None,
     }
     if world == 1 and not args.no_sweep:
@@ -331,6 +348,8 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
         result["strided_variants"] = strided_variants(astra, dev, peak)
         result["decode_chain"] = decode_chain(astra, dev)
         result["fp32_variants"] = fp32_variants(astra, dev, peak)
+        result["rmsnorm_cost_model"] = rmsnorm_cost_model(astra, dev, peak)
+        result["allreduce_rmsnorm"] = allreduce_variants(astra, dev, peak)
     if world == 1 and not args.no_ablation:
         from paper_2509_07506_b200 import ablation
         astra_build.ensure_built(ablation=True)
@@ -340,6 +359,7 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
                               "summary": abl["summary"], "rows": abl["rows"], "timing": abl["timing"]}
     if world == 1 and not args.no_cpu:
         result["cpu_baseline"] = oracle_baseline(cfg, rows=min(args.cpu_rows, T))
+        result["cpu_baseline"]["gpu_vs_oracle"] = oracle_agreement(astra, cfg, dev, rows=min(256, T))
     return result
 
 
@@ -422,7 +442,10 @@ def shape_sweep(astra, dev, peak) -> list:
         best = cold if big else row["us_cold_graph"]
         gbs = nbytes / (best * 1e-6) / 1e9
         row["gbs_cold"] = round(gbs, 1)
-        row["frac_of_measured_peak"] = round(gbs / peak, 4) if big else None
+        if big:
+            row.update(fractions(gbs, peak))
+        else:
+            row["frac_of_measured_peak"] = None
         rows.append(row)
 
     def rms(dtype, T, H):
@@ -472,9 +495,87 @@ def decode_chain(astra, dev) -> list:
             astra.astra_silu_and_mul(so, si)
             astra.astra_merge_attn_states_lse(vo, lo, va, sa, vb, sb)
 
+        prepared = [astra.prepare_fused_add_rmsnorm(x, r, w, 1e-5), astra.prepare_silu_and_mul(so, si),
+                    astra.prepare_merge_attn_states_lse(vo, lo, va, sa, vb, sb)]
+
+        def step_prepared(_=None):
+            for call in prepared:
+                call()
+
         eager = _time_launches(step)
+        ready = _time_launches(step_prepared)
         graph = _time_graph(step, [None], launches=20)
-        rows.append({"tokens": T, "us_per_step_eager": round(eager, 2), "us_per_step_graph": round(graph, 2)})
+        rows.append({"tokens": T, "us_per_step_eager": round(eager, 2), "us_per_step_prepared": round(ready, 2),
+                     "us_per_step_graph": round(graph, 2)})
+    return rows
+
+
+def rmsnorm_cost_model(astra, dev, peak) -> list:
+    """fused_add_rmsnorm, bf16: device time (CUDA graph of 100 launches, L2-cold) at seven token counts
+    per hidden size, and the least-squares fit t = t0 + bytes / BW over them.  t0 is the fixed cost of
+    a launch (ramp-up and drain of the grid, with the launch itself overlapped by the previous kernel's
+    tail); BW is the streaming rate once the grid is in flight.  A mid-size shape's fraction of the
+    peak is bytes / (t0 + bytes / BW) / peak: what is lost there is t0, not streaming rate."""
+    td = torch.bfloat16
+    out = []
+    for H in wl.SWEEP_H:
+        pts = []
+        for T in (256, 512, 1024, 2048, 4096, 8192, 16384):
+            nbytes = wl.rmsnorm_bytes(T, H)
+            make = lambda: (torch.randn((T, H), device=dev).to(td), torch.randn((T, H), device=dev).to(td),  # noqa: E731
+                            torch.ones((H,), device=dev, dtype=td))
+            sets = [make()] if nbytes > 2 * L2_BYTES else _rotating(make, nbytes)
+            us = _time_graph(lambda b: astra.astra_fused_add_rmsnorm(b[0], b[1], b[2], 1e-5), sets)
+            pts.append((T, nbytes, us))
+            del sets
+        n = len(pts)
+        sx = sum(p[1] for p in pts); sy = sum(p[2] for p in pts)
+        sxx = sum(p[1] * p[1] for p in pts); sxy = sum(p[1] * p[2] for p in pts)
+        slope = (n * sxy - sx * sy) / (n * sxx - sx * sx)      # us per byte
+        t0 = (sy - slope * sx) / n
+        bw = 1e-3 / slope                                      # GB/s
+        out.append({"H": H, "t0_us": round(t0, 2), "bw_gbs": round(bw, 1), "bw_frac_of_measured_peak": round(bw / peak, 4),
+                    "points": [{"T": T, "us": round(us, 2), "gbs": round(b / us / 1e3, 1),
+                                "frac_of_measured_peak": round(b / us / 1e3 / peak, 4),
+                                "model_us": round(t0 + slope * b, 2)} for T, b, us in pts]})
+    return out
+
+
+def allreduce_variants(astra, dev, peak) -> list:
+    """astra_fused_allreduce_add_rmsnorm (the partial hidden states of N tensor-parallel ranks summed
+    inside add + RMSNorm) with all partials in this GPU's memory: (N + 3) * T * H * 2 algorithmic bytes
+    against the HBM roofline at the prefill shape, device microseconds at decode shapes, and beside each
+    the separate-kernels route it replaces on one GPU (N - 1 torch adds, then astra_fused_add_rmsnorm).
+    Over NVLink the partials of the other ranks would arrive at link speed instead; not measured here."""
+    td = torch.bfloat16
+    rows = []
+    H = wl.CHAIN_H
+    for T in (wl.CHAIN_T, 1024, 16):
+        for n in (2, 4, 8):
+            nbytes = wl.allreduce_rmsnorm_bytes(T, H, n)
+            make = lambda: ([torch.randn((T, H), device=dev).to(td) for _ in range(n)], torch.randn((T, H), device=dev).to(td),  # noqa: E731
+                            torch.empty((T, H), device=dev, dtype=td), torch.ones((H,), device=dev, dtype=td))
+            big = nbytes > 2 * L2_BYTES
+            sets = [make()] if big else _rotating(make, nbytes)
+            fused = lambda b: astra.astra_fused_allreduce_add_rmsnorm(b[2], b[1], b[0], b[3], 1e-5)  # noqa: E731
+
+            def separate(b):
+                acc = b[2]
+                torch.add(b[0][0], b[0][1], out=acc)
+                for p in b[0][2:]:
+                    acc.add_(p)
+                astra.astra_fused_add_rmsnorm(acc, b[1], b[3], 1e-5)
+
+            us = _time_graph(fused, sets)
+            us_sep = _time_graph(separate, sets)
+            gbs = nbytes / us / 1e3
+            row = {"shape": [T, H], "n_parts": n, "algorithmic_bytes": nbytes, "us_device": round(us, 2),
+                   "gbs": round(gbs, 1), "us_device_separate_kernels": round(us_sep, 2),
+                   "speedup_over_separate_kernels": round(us_sep / us, 2)}
+            if big:
+                row.update(fractions(gbs, peak))
+            rows.append(row)
+            del sets
     return rows
 
 
@@ -488,8 +589,7 @@ def strided_variants(astra, dev, peak) -> list:
     def add(name, nbytes, fn):
         us = _time_launches(fn)
         gbs = nbytes / (us * 1e-6) / 1e9
-        rows.append({"call": name, "us_per_call": round(us, 2), "gbs": round(gbs, 1),
-                     "frac_of_measured_peak": round(gbs / peak, 4)})
+        rows.append({"call": name, "us_per_call": round(us, 2), "gbs": round(gbs, 1), **fractions(gbs, peak)})
 
     x = torch.randn((T, H), device=dev).to(bf); r = torch.randn((T, H), device=dev).to(bf)
     y = torch.empty_like(x); ro = torch.empty_like(x); w = torch.ones((H,), device=dev, dtype=bf)
@@ -522,8 +622,7 @@ def fp32_variants(astra, dev, peak) -> list:
     def add(name, nbytes, fn):
         us = _time_launches(fn)
         gbs = nbytes / (us * 1e-6) / 1e9
-        rows.append({"call": name, "us_per_call": round(us, 2), "gbs": round(gbs, 1),
-                     "frac_of_measured_peak": round(gbs / peak, 4)})
+        rows.append({"call": name, "us_per_call": round(us, 2), "gbs": round(gbs, 1), **fractions(gbs, peak)})
 
     x = torch.randn((T, H), device=dev); r = torch.randn((T, H), device=dev); w = torch.ones((H,), device=dev)
     add("astra_fused_add_rmsnorm fp32 [8192,4096]", wl.rmsnorm_bytes(T, H, 4),
@@ -541,9 +640,10 @@ def fp32_variants(astra, dev, peak) -> list:
 
 
 def table4_sweep(astra, dev, peak) -> list:
-    """The paper's Table 4 shapes, fp16 (the type its fragments use): device us/call from a CUDA
-    graph, L2-hot and L2-cold, beside the paper's H100 figures (measured inside a serving framework
-    on another machine: context only)."""
+    """The paper's Table 4 shapes, fp16 (the type its fragments use): us/call through the binding
+    (`us_eager`: every argument checked and converted per call; `us_prepared`: a prepared call
+    re-issued), device us/call from a CUDA graph, L2-hot and L2-cold, beside the paper's H100 figures
+    (measured inside a serving framework on another machine: context only)."""
     rows = []
     td = torch.float16
     for kernel, shape, h100_base, h100_opt in wl.TABLE4:
@@ -554,21 +654,26 @@ def table4_sweep(astra, dev, peak) -> list:
                             torch.randn((T, Hh, Dh), device=dev).to(td), torch.rand((T, Hh), device=dev) * 20 - 5,
                             torch.randn((T, Hh, Dh), device=dev).to(td), torch.rand((T, Hh), device=dev) * 20 - 5)
             call = lambda b: astra.astra_merge_attn_states_lse(b[0], b[1], b[2], b[3], b[4], b[5])  # noqa: E731
+            prep = lambda b: astra.prepare_merge_attn_states_lse(b[0], b[1], b[2], b[3], b[4], b[5])  # noqa: E731
         elif kernel == "fused_add_rmsnorm":
             T, H = shape
             nbytes = wl.rmsnorm_bytes(T, H)
             make = lambda: (torch.randn((T, H), device=dev).to(td), torch.randn((T, H), device=dev).to(td),  # noqa: E731
                             torch.ones((H,), device=dev, dtype=td))
             call = lambda b: astra.astra_fused_add_rmsnorm(b[0], b[1], b[2], 1e-6)  # noqa: E731
+            prep = lambda b: astra.prepare_fused_add_rmsnorm(b[0], b[1], b[2], 1e-6)  # noqa: E731
         else:
             T, D = shape
             nbytes = wl.silu_bytes(T, D)
             make = lambda: (torch.empty((T, D), device=dev, dtype=td), (2 * torch.randn((T, 2 * D), device=dev)).to(td))  # noqa: E731
             call = lambda b: astra.astra_silu_and_mul(b[0], b[1])  # noqa: E731
+            prep = lambda b: astra.prepare_silu_and_mul(b[0], b[1])  # noqa: E731
         one = [make()]
         many = _rotating(make, nbytes)
+        ready = prep(one[0])
         rows.append({"kernel": kernel, "dtype": "fp16", "shape": list(shape), "algorithmic_bytes": nbytes,
                      "us_eager": round(_time_sets(call, one), 2),
+                     "us_prepared": round(_time_launches(ready), 2),
                      "us_hot_graph": round(_time_graph(call, one), 2),
                      "us_cold_graph": round(_time_graph(call, many), 2),
                      "paper_h100_us_base": h100_base, "paper_h100_us_opt": h100_opt})
@@ -611,7 +716,52 @@ def oracle_baseline(cfg, rows: int) -> dict:
             "seconds": round(sec, 3)}
 
 
-def run_reference(args, rank: int) -> dict | None:
+def oracle_agreement(astra, cfg, dev, rows: int) -> dict:
+    """Part of the CPU-baseline leg: the library's outputs on the first `rows` rows of the three chain
+    calls against the oracle's, as the largest error in units of the storage type's spacing at the
+    oracle's value (bf16 here; 0.5 is a correctly rounded result), the score error in absolute terms,
+    and whether the residual sum agrees bit for bit."""
+    import numpy as np
+    import oracle
+    rms, silu, merge = cfg["rmsnorm"], cfg["silu"], cfg["merge"]
+
+    def spacing(v):
+        _, e = np.frexp(np.abs(v))
+        return np.ldexp(1.0, np.maximum(e - 1, -126) - 7)
+
+    def worst(gpu, want):
+        gpu = gpu.cpu().to(torch.float64).numpy()
+        nz = want != 0
+        return round(float(np.max(np.abs(gpu - want)[nz] / spacing(want[nz]))), 3)
+
+    x, r, w = rms.x[:rows].to(dev), rms.residual[:rows].to(dev), rms.weight.to(dev)
+    astra.astra_fused_add_rmsnorm(x, r, w, rms.eps)
+    oy, orr = oracle.fused_add_rmsnorm(wl.bits(rms.x[:rows]), wl.bits(rms.residual[:rows]), wl.bits(rms.weight),
+                                       rms.eps, rms.dtype)
+    si = silu.input[:rows].to(dev)
+    so = torch.empty((rows, si.shape[1] // 2), dtype=si.dtype, device=dev)
+    astra.astra_silu_and_mul(so, si)
+    osilu = oracle.silu_and_mul(wl.bits(silu.input[:rows]), silu.dtype)
+    va, vb = merge.v_a[:rows].to(dev), merge.v_b[:rows].to(dev)
+    sa, sb = merge.lse_a[:rows].to(dev), merge.lse_b[:rows].to(dev)
+    vo, lo = torch.empty_like(va), torch.empty_like(sa)
+    astra.astra_merge_attn_states_lse(vo, lo, va, sa, vb, sb)
+    ov, ol = oracle.merge_attn_states_lse(wl.bits(merge.v_a[:rows]), merge.lse_a[:rows].numpy(),
+                                          wl.bits(merge.v_b[:rows]), merge.lse_b[:rows].numpy(), merge.dtype)
+    torch.cuda.synchronize()
+    return {"rows": rows, "max_err_ulp": {"fused_add_rmsnorm": worst(x, oy), "silu_and_mul": worst(so, osilu),
+                                          "merge_attn_states_lse": worst(vo, ov)},
+            "residual_sum_bit_exact": bool(np.array_equal(wl.bits(r.cpu()), orr)),
+            "max_lse_abs_err": float(np.max(np.abs(lo.cpu().to(torch.float64).numpy() - ol)))}
+
+
+def chain_workload_name(T: int) -> str:
+    return (f"configs[4]: Llama-3-8B prefill-shaped chain, T={T} per GPU, bf16: "
+            f"fused_add_rmsnorm [{T},4096] -> silu_and_mul [{T},2*14336] -> "
+            f"merge_attn_states_lse [{T},32,128]")
+
+
+def run_reference(args, rank: int, world: int) -> dict | None:
     if rank != 0:
         return None
     import oracle
@@ -633,14 +783,14 @@ def run_reference(args, rank: int) -> dict | None:
     sec = time.perf_counter() - t0
     b = sum(chain_bytes(rows).values())
     value = round(b * args.steps / sec / 1e9, 3)
-    sample = (f"each step = the fp64 oracle over the first {rows} of 8192 rows/tokens of the three chain calls, "
+    sample = (f"each step = the fp64 oracle over the first {rows} of {wl.CHAIN_T} rows/tokens of the three chain calls, "
               f"OpenMP over rows on {cores} host cores")
     return {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": max(args.gpus, world),
+        "launcher": os.environ.get("ASTRA_BENCH_LAUNCHER", "external launcher" if world > 1 else "single process"),
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(sec / args.steps * 1e3, 3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "configs[4]: Llama-3-8B prefill-shaped chain (bounded sample of T=8192), bf16 storage",
-                   "sample": sample, "seed": 4},
+        "config": {"workload": chain_workload_name(wl.CHAIN_T), "sample": sample, "seed": 4},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -670,10 +820,20 @@ def main() -> int:
     if args.warmup < 3:
         args.warmup = 3
 
+    # `python bench.py --gpus N` without a launcher: start the N ranks of this node here (one process
+    # per GPU, rendezvous over 127.0.0.1); under torchrun the ranks already exist.
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        if args.impl == "astra" and args.backend == "nccl" and torch.cuda.device_count() < args.gpus:
+            print(f"bench.py: --gpus {args.gpus} needs {args.gpus} GPUs, this machine has {torch.cuda.device_count()}",
+                  file=sys.stderr)
+            return 1
+        os.environ["ASTRA_BENCH_LAUNCHER"] = "self-spawned ranks"
+        return multi.spawn_ranks([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], args.gpus)
+
     rank, world, local_rank = multi.env_rank_world()
 
     if args.impl == "reference":
-        res = run_reference(args, rank)
+        res = run_reference(args, rank, world)
         if res is not None:
             print(json.dumps(res), flush=True)
         return 0

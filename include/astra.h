@@ -158,6 +158,35 @@ astra_status_t astra_merge_attn_states_lse_ex(void *v_out, float *lse_out,
                                               const int64_t *strides,
                                               astra_dtype_t dtype, void *cuda_stream);
 
+/*
+ * fused_allreduce_add_rmsnorm: fused_add_rmsnorm (Table 1, Kernel 2) on a hidden state that arrives
+ * as n_parts partial sums, one per tensor-parallel rank -- the all-reduce that precedes Kernel 2 in
+ * tensor-parallel serving, folded into it (the paper's per-shape study, Table 4, shows these small
+ * calls bound by fixed cost rather than bandwidth; the paper itself states Kernel 2 for one x only):
+ *     x = x_0 + x_1 + ... + x_{n-1};  s = x + r;  residual <- s;  y = s / sqrt(mean(s^2) + eps) (.) w
+ *
+ *   y        [T, H]  out.
+ *   residual [T, H]  in: r.  out: s rounded once to the storage type  (updated in place)
+ *   x_parts  HOST array of n_parts device pointers, in rank order, each a dense [T, H] tensor.
+ *            A partial may live in another GPU's memory if that memory is mapped into this
+ *            process (peer access): the kernel reads it with ordinary per-thread loads only.
+ *   n_parts  1 .. 16 (else ASTRA_ERR_BAD_SHAPE).  n_parts = 1 computes exactly what
+ *            astra_fused_add_rmsnorm_ex computes with separate y.
+ *   weight   [H].
+ *
+ * Arithmetic: every addition is one binary32 addition; the partials are added in rank order
+ * starting from x_0 and the residual is added last; nothing is rounded to the storage type before
+ * that.  Ranks that run this on the same partials therefore produce identical bits.
+ * Ordering: the call waits for nothing.  The caller must order it after every rank has finished
+ * writing its partial, and must keep the partials unchanged until the kernel has completed.
+ * y and residual must not overlap each other, any partial, or weight (ASTRA_ERR_OVERLAP); the
+ * partials may overlap one another.  Every pointer needs the alignment of its element.
+ */
+astra_status_t astra_fused_allreduce_add_rmsnorm(void *y, void *residual,
+                                                 const void *const *x_parts, int32_t n_parts,
+                                                 const void *weight, int64_t T, int64_t H, float eps,
+                                                 astra_dtype_t dtype, void *cuda_stream);
+
 /* Static, NUL-terminated description of a status code (never NULL). */
 const char *astra_status_string(astra_status_t status);
 

@@ -6,7 +6,13 @@ load the library; the first call does, and fails loudly if it has not been built
 """
 from .binding import (  # noqa: F401
     AstraError,
+    PreparedCall,
     astra_fused_add_rmsnorm,
+    astra_fused_allreduce_add_rmsnorm,
+    prepare_fused_add_rmsnorm,
+    prepare_fused_allreduce_add_rmsnorm,
+    prepare_merge_attn_states_lse,
+    prepare_silu_and_mul,
     astra_fused_add_rmsnorm_ex,
     astra_merge_attn_states_lse,
     astra_merge_attn_states_lse_ex,

@@ -35,6 +35,7 @@ EXPORTED_SYMBOLS = (
     "astra_fused_add_rmsnorm_ex",
     "astra_silu_and_mul_ex",
     "astra_merge_attn_states_lse_ex",
+    "astra_fused_allreduce_add_rmsnorm",
     "astra_status_string",
     "astra_build_id",
 )
@@ -75,6 +76,8 @@ def load_library() -> ctypes.CDLL:
     lib.astra_merge_attn_states_lse_ex.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64,
                                                    ctypes.POINTER(ctypes.c_int64), i32, vp]
     lib.astra_merge_attn_states_lse_ex.restype = i32
+    lib.astra_fused_allreduce_add_rmsnorm.argtypes = [vp, vp, ctypes.POINTER(vp), i32, vp, i64, i64, f32, i32, vp]
+    lib.astra_fused_allreduce_add_rmsnorm.restype = i32
     lib.astra_status_string.argtypes = [i32]
     lib.astra_status_string.restype = ctypes.c_char_p
     lib.astra_build_id.argtypes = []
@@ -273,6 +276,39 @@ def astra_merge_attn_states_lse(v_out: torch.Tensor, lse_out: Optional[torch.Ten
                                 stream: Optional[torch.cuda.Stream] = None) -> None:
     """v_out, lse_out <- merge of (v_a, lse_a) and (v_b, lse_b).  v_* [T, Hh, D]; lse_* [T, Hh] fp32."""
     prepare_merge_attn_states_lse(v_out, lse_out, v_a, lse_a, v_b, lse_b)(stream)
+
+
+def prepare_fused_allreduce_add_rmsnorm(y: torch.Tensor, residual: torch.Tensor, parts, weight: torch.Tensor,
+                                        eps: float) -> PreparedCall:
+    """Validated, re-issuable form of :func:`astra_fused_allreduce_add_rmsnorm`."""
+    parts = list(parts)
+    _check(y, "y")
+    code = _code(y, "y")
+    if y.dim() != 2:
+        raise ValueError("y must be [T, H]")
+    T, H = y.shape
+    _check(residual, "residual", y.dtype, (T, H), y.device)
+    _check(weight, "weight", y.dtype, (H,), y.device)
+    if not 1 <= len(parts) <= 16:
+        raise ValueError(f"between 1 and 16 partial hidden states are supported, got {len(parts)}")
+    for i, p in enumerate(parts):
+        # a partial may sit on another GPU (that is the point of the call): no device check here
+        _check(p, f"parts[{i}]", y.dtype, (T, H))
+    table = (ctypes.c_void_p * len(parts))(*[p.data_ptr() for p in parts])
+    args = (_ptr(y), _ptr(residual), table, ctypes.c_int(len(parts)), _ptr(weight), ctypes.c_int64(T),
+            ctypes.c_int64(H), ctypes.c_float(float(eps)), ctypes.c_int(code))
+    return PreparedCall("astra_fused_allreduce_add_rmsnorm", load_library().astra_fused_allreduce_add_rmsnorm,
+                        args, y.device, (y, residual, weight, table, *parts))
+
+
+def astra_fused_allreduce_add_rmsnorm(y: torch.Tensor, residual: torch.Tensor, parts, weight: torch.Tensor,
+                                      eps: float, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """y <- RMSNorm(sum(parts) + residual) * weight, residual <- sum(parts) + residual (in place).
+    ``parts`` is the sequence of per-rank partial hidden states [T, H], in rank order; they are added
+    in that order in binary32 and the residual last.  The partials may live on other GPUs whose
+    memory this process can address; y, residual and weight live on the GPU that runs the kernel.
+    The call waits for nothing: order it after the partials have been written."""
+    prepare_fused_allreduce_add_rmsnorm(y, residual, parts, weight, eps)(stream)
 
 
 # ---- strided / out-of-place forms ---------------------------------------------------------------

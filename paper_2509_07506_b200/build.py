@@ -19,13 +19,14 @@ INCLUDE = os.path.join(ROOT, "include")
 LIB_PATH = os.path.join(PKG_DIR, "libastra.so")
 ABLATION_LIB_PATH = os.path.join(PKG_DIR, "libastra_ablation.so")
 
-SOURCES = ["astra.cu"]
+SOURCES = ["astra.cu", "astra_allreduce.cu"]
 ABLATION_SOURCES = ["ablation.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
     "-O3", "-std=c++17", "-lineinfo",
     "-Xcompiler", "-fPIC", "-shared",
     "-cudart", "static",
+    "--threads", "0",
 ]
 
 

@@ -1,0 +1,157 @@
+// C ABI of astra_fused_allreduce_add_rmsnorm (declared in astra.h): argument validation, launch-shape
+// selection and the kernel launch.  Same conventions as the rest of the library: nothing is
+// allocated, nothing synchronises, errors are status codes.
+#include <cuda_runtime.h>
+
+#include "astra.h"
+#include "fused_allreduce_add_rmsnorm.cuh"
+#include "launch.cuh"
+
+namespace {
+
+using namespace astra;
+using namespace astra::host;
+
+inline int round_up_to(int v, int m) { return (v + m - 1) / m * m; }
+
+// Register-resident rows hold at most 32 16-bit units per thread in vectors of 8 or 16 bytes.
+// UVEC is the vector width in units, VPT the vectors per thread.
+template <int DT, int UVEC, int VPT, int GROUP>
+cudaError_t launch_reg(const AllreduceOperands &op, const uint16_t *w, unsigned rows, int threads, int H,
+                       float eps, float inv_H, cudaStream_t stream) {
+    if constexpr (UVEC >= 4 && UVEC >= Storage<DT>::UNITS && UVEC * VPT <= 32)
+        return launch(fused_allreduce_add_rmsnorm_reg_kernel<DT, UVEC / Storage<DT>::UNITS, VPT, GROUP>, rows,
+                      threads, stream, op, w, H, eps, inv_H);
+    return cudaErrorInvalidValue;
+}
+
+// Per-thread share of a register-resident row for a given width, or 0 if the row does not fit:
+// start at 8 units (one 16-byte vector) when four partials are in flight per vector and at 16
+// otherwise; double it while the block would exceed what the register file allows; halve it while
+// the block would fall under 128 threads.
+template <int UVEC, int GROUP>
+inline int pick_vpt(int nvec, int *threads_out) {
+    if (UVEC < 4) return 0;  // 2- and 4-byte vectors take the two-sweep kernel
+    constexpr int kMaxVpt = 32 / (UVEC < 4 ? 4 : UVEC);
+    auto threads_for = [&](int v) { return round_up_to((nvec + v - 1) / v, 32); };
+    int vpt = (GROUP >= 4 ? 8 : 16) / UVEC;
+    if (vpt < 1) vpt = 1;
+    while (vpt <= kMaxVpt && threads_for(vpt) > allreduce_reg_max_threads(UVEC * vpt, GROUP)) vpt <<= 1;
+    if (vpt > kMaxVpt) return 0;
+    while (vpt > 1 && threads_for(vpt) < 128) vpt >>= 1;
+    *threads_out = threads_for(vpt);
+    return vpt;
+}
+
+// Launches over all rows (split where the grid limit requires).  vpt = 0 selects the two-sweep kernel.
+template <int DT, int UVEC, int GROUP>
+cudaError_t launch_rows(AllreduceOperands op, const uint16_t *w, int64_t T, int H, float eps, int vpt,
+                        int threads, cudaStream_t stream) {
+  if constexpr (UVEC >= Storage<DT>::UNITS) {
+    constexpr int VEC = UVEC / Storage<DT>::UNITS;
+    const int nvec = H / VEC;
+    const float inv_H = 1.0f / static_cast<float>(H);
+    const int sweep_iters = (nvec + 1023) / 1024;
+    const int sweep_threads = round_up_to((nvec + sweep_iters - 1) / sweep_iters, 32);
+    const int64_t row_units = static_cast<int64_t>(H) * Storage<DT>::UNITS;
+    const int64_t rows_per_launch = kMaxRowsPerLaunch;
+    for (int64_t t0 = 0; t0 < T; t0 += rows_per_launch) {
+        const unsigned rows = static_cast<unsigned>(T - t0 < rows_per_launch ? T - t0 : rows_per_launch);
+        AllreduceOperands o = op;
+        for (int p = 0; p < op.n_parts; ++p) o.part[p] += t0 * row_units;
+        o.r += t0 * row_units;
+        o.y += t0 * row_units;
+        o.r_out += t0 * row_units;
+        cudaError_t err;
+        switch (vpt) {
+            case 0: err = launch(fused_allreduce_add_rmsnorm_twopass_kernel<DT, VEC, GROUP>, rows, sweep_threads,
+                                 stream, o, w, H, eps, inv_H); break;
+            case 1: err = launch_reg<DT, UVEC, 1, GROUP>(o, w, rows, threads, H, eps, inv_H, stream); break;
+            case 2: err = launch_reg<DT, UVEC, 2, GROUP>(o, w, rows, threads, H, eps, inv_H, stream); break;
+            case 4: err = launch_reg<DT, UVEC, 4, GROUP>(o, w, rows, threads, H, eps, inv_H, stream); break;
+            default: err = launch_reg<DT, UVEC, 8, GROUP>(o, w, rows, threads, H, eps, inv_H, stream); break;
+        }
+        if (err != cudaSuccess) return err;
+    }
+  }
+  return cudaSuccess;
+}
+
+// Four partial loads in flight per vector when there are more than two partials and the row still
+// fits the registers that way; otherwise two.
+template <int DT, int UVEC>
+cudaError_t choose_group(const AllreduceOperands &op, const uint16_t *w, int64_t T, int H, float eps,
+                         cudaStream_t stream) {
+  if constexpr (UVEC >= Storage<DT>::UNITS) {
+    const int nvec = H / (UVEC / Storage<DT>::UNITS);
+    int threads = 0;
+    if (op.n_parts > 2) {
+        const int vpt4 = pick_vpt<UVEC, 4>(nvec, &threads);
+        if (vpt4 > 0 || UVEC < 4) return launch_rows<DT, UVEC, 4>(op, w, T, H, eps, vpt4, threads, stream);
+    }
+    const int vpt2 = pick_vpt<UVEC, 2>(nvec, &threads);
+    if (vpt2 > 0 || op.n_parts <= 2) return launch_rows<DT, UVEC, 2>(op, w, T, H, eps, vpt2, threads, stream);
+    return launch_rows<DT, UVEC, 4>(op, w, T, H, eps, 0, 0, stream);  // many partials, very wide row
+  }
+  return cudaErrorInvalidValue;
+}
+
+template <int DT>
+cudaError_t dispatch(const AllreduceOperands &op, const uint16_t *w, int64_t T, int H, float eps,
+                     cudaStream_t stream) {
+    VecPick pick(8);
+    pick.extent(static_cast<int64_t>(H) * Storage<DT>::UNITS).pointer(op.r).pointer(op.y).pointer(op.r_out).pointer(w);
+    for (int p = 0; p < op.n_parts; ++p) pick.pointer(op.part[p]);
+    switch (pick.vec) {
+        case 8: return choose_group<DT, 8>(op, w, T, H, eps, stream);
+        case 4: return choose_group<DT, 4>(op, w, T, H, eps, stream);
+        case 2: return choose_group<DT, 2>(op, w, T, H, eps, stream);
+        default: return choose_group<DT, 1>(op, w, T, H, eps, stream);
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+astra_status_t astra_fused_allreduce_add_rmsnorm(void *y, void *residual, const void *const *x_parts,
+                                                 int32_t n_parts, const void *weight, int64_t T, int64_t H,
+                                                 float eps, astra_dtype_t dtype, void *cuda_stream) {
+    if (!valid_dtype(dtype)) return ASTRA_ERR_BAD_DTYPE;
+    const int64_t U = units_per_elem(dtype);
+    if (n_parts < 1 || n_parts > kMaxParts) return ASTRA_ERR_BAD_SHAPE;
+    if (T < 0 || H <= 0 || H > kMaxRowUnits / U) return ASTRA_ERR_BAD_SHAPE;
+    if (T > 0 && H > kInt64Max / 4 / T) return ASTRA_ERR_BAD_SHAPE;
+    if (T == 0) return ASTRA_OK;
+    if (!y || !residual || !x_parts || !weight) return ASTRA_ERR_NULL_POINTER;
+    for (int p = 0; p < n_parts; ++p)
+        if (!x_parts[p]) return ASTRA_ERR_NULL_POINTER;
+    const size_t eb = static_cast<size_t>(2 * U);
+    if (!aligned(y, eb) || !aligned(residual, eb) || !aligned(weight, eb)) return ASTRA_ERR_MISALIGNED;
+    for (int p = 0; p < n_parts; ++p)
+        if (!aligned(x_parts[p], eb)) return ASTRA_ERR_MISALIGNED;
+    // The two outputs overlap nothing else.  (A partial in another GPU's memory has an address in
+    // the same unified space, so the byte-range test is meaningful for it too.)  Partials may
+    // overlap one another: they are only read.
+    const int64_t bytes = T * H * U * 2, wbytes = H * U * 2;
+    if (overlaps(y, bytes, residual, bytes) || overlaps(y, bytes, weight, wbytes) ||
+        overlaps(residual, bytes, weight, wbytes))
+        return ASTRA_ERR_OVERLAP;
+    for (int p = 0; p < n_parts; ++p)
+        if (overlaps(y, bytes, x_parts[p], bytes) || overlaps(residual, bytes, x_parts[p], bytes))
+            return ASTRA_ERR_OVERLAP;
+    AllreduceOperands op;
+    for (int p = 0; p < kMaxParts; ++p)
+        op.part[p] = static_cast<const uint16_t *>(x_parts[p < n_parts ? p : 0]);
+    op.n_parts = n_parts;
+    op.r = static_cast<const uint16_t *>(residual);
+    op.r_out = static_cast<uint16_t *>(residual);
+    op.y = static_cast<uint16_t *>(y);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const uint16_t *wp = static_cast<const uint16_t *>(weight);
+    cudaError_t err = cudaSuccess;
+    ASTRA_FOR_DTYPE(dtype, err = dispatch<DT>(op, wp, T, static_cast<int>(H), eps, stream));
+    return launch_status(err);
+}
+
+}  // extern "C"

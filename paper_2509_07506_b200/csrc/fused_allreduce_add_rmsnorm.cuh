@@ -1,0 +1,215 @@
+// fused_allreduce_add_rmsnorm: fused_add_rmsnorm (Astra paper, Table 1, Kernel 2) on a hidden state
+// that arrives as N partial sums, one per tensor-parallel rank:
+//     x = x_0 + x_1 + ... + x_{N-1};   s = x + r;   r_out <- s;   y <- s / sqrt(mean(s^2) + eps) * w
+// Every addition is one binary32 addition, in rank order, the residual last, so that all ranks of a
+// group that run this on the same partials produce identical bits.
+//
+// This is the "one-shot" all-reduce: each rank reads all N partials of the rows it normalises (its
+// own from local memory, the others through peer-mapped addresses) and never writes to a peer.
+// All loads are plain per-thread `ld.global` (no multicast, no bulk or tensor-map copies), so a
+// partial may live in another GPU's memory.  The kernel waits for nothing: the caller orders it
+// after every rank has finished writing its partial (stream events, a host barrier).
+//
+// HBM/NVLink-bound: (N + 3) * 2 bytes per element of 16-bit storage (N partials and r read, y and
+// r_out written).  One block owns a row and keeps the running binary32 sums in registers; the
+// partials are fetched GROUP at a time so that GROUP (+1 for the residual) vector loads per thread
+// are in flight before the first addition.
+#pragma once
+
+#include "fused_add_rmsnorm.cuh"
+
+namespace astra {
+
+constexpr int kMaxParts = 16;
+
+// Dense [T, H] operands (row pitch = H).  Pointers are in 16-bit units.  r_out may be exactly r
+// (each thread reads the residual vectors it later overwrites); y overlaps nothing.
+struct AllreduceOperands {
+    const uint16_t *part[kMaxParts];  // rank order
+    const uint16_t *r;
+    uint16_t *y;
+    uint16_t *r_out;
+    int n_parts;
+};
+
+// s += x, two elements per instruction where the vector length is even (same roundings as scalar adds).
+template <int VEC>
+__device__ __forceinline__ void accumulate(float (&s)[VEC], const float (&x)[VEC]) {
+    if constexpr (VEC % 2 == 0) {
+#pragma unroll
+        for (int k = 0; k < VEC; k += 2) {
+            const float2 t = __fadd2_rn(make_float2(s[k], s[k + 1]), make_float2(x[k], x[k + 1]));
+            s[k] = t.x;
+            s[k + 1] = t.y;
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) s[k] += x[k];
+    }
+}
+
+// Largest block of the register-resident kernel: a thread holds its share of the row as binary32 sums
+// (one register per element) plus GROUP + 1 packed input copies of it, and the register file is
+// 64 K registers per block.  `units` = 16-bit units of the row per thread.
+__host__ __device__ constexpr int allreduce_reg_max_threads(int units, int group) {
+    return units <= 8 ? 1024 : (units <= 16 ? 512 : (group <= 2 ? 512 : 256));
+}
+
+// Register-resident row: thread i owns vectors i, i + blockDim.x, ... (at most VPT of them).
+// Requires nvec = H / VEC <= VPT * blockDim.x and blockDim.x <= allreduce_reg_max_threads(...).
+template <int DT, int VEC, int VPT, int GROUP>
+__global__ void __launch_bounds__(allreduce_reg_max_threads(VEC * VPT * Storage<DT>::UNITS, GROUP))
+fused_allreduce_add_rmsnorm_reg_kernel(const __grid_constant__ AllreduceOperands op,
+                                       const uint16_t *__restrict__ weight, int H, float eps, float inv_H) {
+    constexpr int UV = VEC * Storage<DT>::UNITS;  // 16-bit units per vector
+    __shared__ float slots[kMaxWarps];
+    const int nvec = H / VEC;
+    const int64_t row = static_cast<int64_t>(blockIdx.x) * H * Storage<DT>::UNITS;  // first unit of the row
+    const int n = op.n_parts;
+    grid_dependency_wait();
+    grid_launch_dependents();
+
+    // the residual is consumed last but requested first, together with the first group of partials
+    Pack<UV> pr[VPT];
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int v = threadIdx.x + i * blockDim.x;
+        if (v < nvec) pr[i] = load<UV, Ld::Stream>(op.r + row + v * UV);
+    }
+
+    float s[VPT][VEC];
+    for (int p0 = 0; p0 < n; p0 += GROUP) {
+        Pack<UV> px[GROUP][VPT];
+#pragma unroll
+        for (int g = 0; g < GROUP; ++g) {
+            if (p0 + g < n) {
+                const uint16_t *base = op.part[p0 + g] + row;
+#pragma unroll
+                for (int i = 0; i < VPT; ++i) {
+                    const int v = threadIdx.x + i * blockDim.x;
+                    if (v < nvec) px[g][i] = load<UV, Ld::Stream>(base + v * UV);
+                }
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < GROUP; ++g) {
+            if (p0 + g < n) {
+#pragma unroll
+                for (int i = 0; i < VPT; ++i) {
+                    const int v = threadIdx.x + i * blockDim.x;
+                    if (v < nvec) {
+                        float fx[VEC];
+                        widen<DT, VEC>(px[g][i], fx);
+                        if (p0 + g == 0) {
+#pragma unroll
+                            for (int k = 0; k < VEC; ++k) s[i][k] = fx[k];
+                        } else {
+                            accumulate(s[i], fx);  // rank order: partial p0 + g joins the sum of those before it
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    float acc = 0.f;
+    float2 acc2 = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int v = threadIdx.x + i * blockDim.x;
+        if (v < nvec) {
+            float fr[VEC];
+            widen<DT, VEC>(pr[i], fr);
+            add_and_square(s[i], fr, s[i], acc, acc2);  // the residual joins last
+            store<UV, St::Stream>(op.r_out + row + v * UV, narrow<DT, VEC>(s[i]));
+        }
+    }
+
+    Pack<UV> pw[VPT];
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int v = threadIdx.x + i * blockDim.x;
+        if (v < nvec) pw[i] = load<UV, Ld::Keep>(weight + v * UV);
+    }
+    const float total = block_sum(acc + (acc2.x + acc2.y), slots);
+    const float rstd = rsqrtf(fmaf(total, inv_H, eps));
+
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int v = threadIdx.x + i * blockDim.x;
+        if (v < nvec) {
+            float fw[VEC], fy[VEC];
+            widen<DT, VEC>(pw[i], fw);
+            scale(s[i], rstd, fw, fy);
+            store<UV, St::Stream>(op.y + row + v * UV, narrow<DT, VEC>(fy));
+        }
+    }
+}
+
+// The rank-order sum of one vector position, GROUP partial loads in flight at a time.
+template <int DT, int VEC, int GROUP>
+__device__ __forceinline__ void rank_order_sum(const AllreduceOperands &op, int64_t at, float (&s)[VEC]) {
+    constexpr int UV = VEC * Storage<DT>::UNITS;
+    const int n = op.n_parts;
+    const Pack<UV> pr = load<UV, Ld::Stream>(op.r + at);
+    for (int p0 = 0; p0 < n; p0 += GROUP) {
+        Pack<UV> px[GROUP];
+#pragma unroll
+        for (int g = 0; g < GROUP; ++g)
+            if (p0 + g < n) px[g] = load<UV, Ld::Stream>(op.part[p0 + g] + at);
+#pragma unroll
+        for (int g = 0; g < GROUP; ++g) {
+            if (p0 + g < n) {
+                float fx[VEC];
+                widen<DT, VEC>(px[g], fx);
+                if (p0 + g == 0) {
+#pragma unroll
+                    for (int k = 0; k < VEC; ++k) s[k] = fx[k];
+                } else {
+                    accumulate(s, fx);
+                }
+            }
+        }
+    }
+    float fr[VEC];
+    widen<DT, VEC>(pr, fr);
+    accumulate(s, fr);
+}
+
+// Any width and any vector size: two sweeps over the row.  The first forms the sums and their
+// squares and writes nothing; the second forms the same sums again (the partials now come from L2
+// where they fit) and writes both outputs, so the in-place residual cannot disturb the reduction.
+template <int DT, int VEC, int GROUP>
+__global__ void __launch_bounds__(1024)
+fused_allreduce_add_rmsnorm_twopass_kernel(const __grid_constant__ AllreduceOperands op,
+                                           const uint16_t *__restrict__ weight, int H, float eps, float inv_H) {
+    constexpr int UV = VEC * Storage<DT>::UNITS;
+    __shared__ float slots[kMaxWarps];
+    const int nvec = H / VEC;
+    const int64_t row = static_cast<int64_t>(blockIdx.x) * H * Storage<DT>::UNITS;
+    grid_dependency_wait();
+    grid_launch_dependents();
+
+    float acc = 0.f;
+    for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
+        float s[VEC];
+        rank_order_sum<DT, VEC, GROUP>(op, row + static_cast<int64_t>(v) * UV, s);
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) acc = fmaf(s[k], s[k], acc);
+    }
+    const float total = block_sum(acc, slots);
+    const float rstd = rsqrtf(fmaf(total, inv_H, eps));
+
+    for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
+        const int64_t at = row + static_cast<int64_t>(v) * UV;
+        float s[VEC], fw[VEC], fy[VEC];
+        rank_order_sum<DT, VEC, GROUP>(op, at, s);
+        widen<DT, VEC>(load<UV, Ld::Keep>(weight + static_cast<int64_t>(v) * UV), fw);
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) fy[k] = s[k] * rstd * fw[k];
+        store<UV, St::Stream>(op.r_out + at, narrow<DT, VEC>(s));
+        store<UV, St::Stream>(op.y + at, narrow<DT, VEC>(fy));
+    }
+}
+
+}  // namespace astra

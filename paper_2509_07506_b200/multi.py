@@ -51,3 +51,82 @@ def max_over_ranks(values: Sequence[float], device: torch.device | str = "cpu") 
 def aggregate_rate(units_per_rank_per_step: float, world: int, steps: int, elapsed_ms: float) -> float:
     """Whole-job rate: units all ranks processed in `steps` steps divided by the (max-over-ranks) time."""
     return world * units_per_rank_per_step * steps / (elapsed_ms * 1e-3)
+
+
+# ---------------------------------------------------------------------------------------------
+# starting the ranks of one node without torchrun
+# ---------------------------------------------------------------------------------------------
+
+def free_port() -> int:
+    import socket
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(argv: Sequence[str], world: int, timeout: float | None = None) -> int:
+    """Run `argv` (a full command line) as `world` processes of one node, one per rank, with the
+    environment a launcher would give them (RANK, LOCAL_RANK, WORLD_SIZE, MASTER_ADDR = 127.0.0.1 and
+    a free MASTER_PORT).  Standard output and error of every rank pass through to this process's.
+    Returns the largest exit code; if a rank fails the others are terminated (they would otherwise
+    wait for it in their next collective)."""
+    import subprocess
+    import time
+    if world < 1:
+        raise ValueError("world must be at least 1")
+    port = free_port()
+    procs = []
+    for rank in range(world):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen(list(argv), env=env))
+    deadline = None if timeout is None else time.time() + timeout
+    worst = 0
+    pending = set(range(world))
+    while pending:
+        for rank in sorted(pending):
+            rc = procs[rank].poll()
+            if rc is None:
+                continue
+            pending.discard(rank)
+            worst = max(worst, abs(rc))
+            if rc != 0:  # the others cannot finish without it
+                for other in pending:
+                    procs[other].terminate()
+        if deadline is not None and time.time() > deadline:
+            for other in pending:
+                procs[other].terminate()
+            worst = max(worst, 124)
+            deadline = None
+        if pending:
+            time.sleep(0.05)
+    return worst
+
+
+# ---------------------------------------------------------------------------------------------
+# tensor-parallel partial hidden states: who reads what in astra_fused_allreduce_add_rmsnorm
+# ---------------------------------------------------------------------------------------------
+
+def exchange_partials(local, export, open_remote, group=None) -> list:
+    """Every rank of a tensor-parallel group holds one partial hidden state; the fused all-reduce
+    kernel of each rank needs all of them, in rank order.  `export(local)` turns this rank's buffer
+    into a picklable handle (for CUDA memory: an inter-process memory handle), the handles are
+    all-gathered over the process group, and `open_remote(handle, owner_rank)` maps every other
+    rank's buffer into this process.  Returns the list of buffers indexed by rank, with this rank's
+    own buffer (not a re-opened copy of it) in its own slot.  Both callables are injected so that the
+    ordering logic is independent of the memory system underneath."""
+    if not (dist.is_available() and dist.is_initialized()):
+        return [local]
+    world, rank = dist.get_world_size(group), dist.get_rank(group)
+    handles = [None] * world
+    dist.all_gather_object(handles, export(local), group=group)
+    return [local if owner == rank else open_remote(handles[owner], owner) for owner in range(world)]
+
+
+def row_block_of_rank(total_rows: int, group=None) -> Tuple[int, int]:
+    """After the fused all-reduce every rank needs the normalised rows it goes on to use.  With
+    sequence-parallel consumers each rank normalises only its own contiguous row block of the
+    [total_rows, H] hidden state (reading that block from all N partials): (first_row, row_count)."""
+    if not (dist.is_available() and dist.is_initialized()):
+        return 0, total_rows
+    return shard_rows(total_rows, dist.get_world_size(group), dist.get_rank(group))

@@ -92,6 +92,27 @@ def rmsnorm_inputs(T: int, H: int, dtype: int = BF16, eps: float = 1e-6, seed: i
     return RmsnormInputs(x, r, w, eps, dtype)
 
 
+@dataclass
+class AllreduceRmsnormInputs:
+    parts: list             # n_parts tensors [T, H], rank order
+    residual: torch.Tensor  # [T, H]
+    weight: torch.Tensor    # [H]
+    eps: float
+    dtype: int
+
+
+def allreduce_rmsnorm_inputs(T: int, H: int, n_parts: int, dtype: int = BF16, eps: float = 1e-5, seed: int = 6,
+                             g: Optional[torch.Generator] = None) -> AllreduceRmsnormInputs:
+    """The per-rank partial hidden states ~ N(0, 1/n_parts) each (so their sum is ~ N(0,1), as the
+    hidden state of the one-GPU operation), then residual ~ N(0,1) and weight ~ N(1, 0.1); drawn in
+    that order."""
+    g = g if g is not None else _gen(seed)
+    parts = [_randn(g, (T, H), dtype, std=float(n_parts) ** -0.5) for _ in range(n_parts)]
+    r = _randn(g, (T, H), dtype)
+    w = _randn(g, (H,), dtype, mean=1.0, std=0.1)
+    return AllreduceRmsnormInputs(parts, r, w, eps, dtype)
+
+
 def silu_inputs(T: int, D: int, dtype: int = BF16, std: float = 2.0, seed: int = 1,
                 g: Optional[torch.Generator] = None) -> SiluInputs:
     """input [T, 2D] ~ N(0, std^2)."""
@@ -205,6 +226,11 @@ def table4_inputs(kernel: str, shape, dtype: int = BF16, seed: int = 5):
 def rmsnorm_bytes(T: int, H: int, elem: int = 2) -> int:
     """Read x and r, write y and r', read the weight once."""
     return 4 * T * H * elem + H * elem
+
+
+def allreduce_rmsnorm_bytes(T: int, H: int, n_parts: int, elem: int = 2) -> int:
+    """Read the n_parts partials and r, write y and r', read the weight once."""
+    return (n_parts + 3) * T * H * elem + H * elem
 
 
 def silu_bytes(T: int, D: int, elem: int = 2) -> int:

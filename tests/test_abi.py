@@ -127,6 +127,44 @@ def test_refused_launch_is_reported_and_stops_the_call(lib):
     assert "launch" in lib.astra_status_string(binding.ASTRA_ERR_CUDA).decode()
 
 
+def test_allreduce_rmsnorm_argument_errors(lib):
+    import ctypes as C
+    f = lib.astra_fused_allreduce_add_rmsnorm
+    Y, R, W = A, 2 * A, 3 * A
+
+    def call(parts=(4 * A, 5 * A), n=None, y=Y, r=R, w=W, T=1, H=8, dtype=0):
+        table = (C.c_void_p * max(1, len(parts)))(*parts) if parts is not None else None
+        return f(y, r, table, len(parts) if n is None else n, w, T, H, 1e-6, dtype, None)
+
+    assert call(y=None) == binding.ASTRA_ERR_NULL_POINTER
+    assert call(r=None) == binding.ASTRA_ERR_NULL_POINTER
+    assert call(w=None) == binding.ASTRA_ERR_NULL_POINTER
+    assert call(parts=None, n=2) == binding.ASTRA_ERR_NULL_POINTER
+    assert call(parts=(4 * A, None)) == binding.ASTRA_ERR_NULL_POINTER
+    assert call(dtype=4) == binding.ASTRA_ERR_BAD_DTYPE
+    assert call(n=0) == binding.ASTRA_ERR_BAD_SHAPE
+    assert call(parts=tuple((4 + i) * A for i in range(17))) == binding.ASTRA_ERR_BAD_SHAPE
+    assert call(T=-1) == binding.ASTRA_ERR_BAD_SHAPE
+    assert call(H=0) == binding.ASTRA_ERR_BAD_SHAPE
+    assert call(H=2 ** 30 + 1) == binding.ASTRA_ERR_BAD_SHAPE
+    assert call(H=2 ** 29 + 1, dtype=binding.ASTRA_FP32) == binding.ASTRA_ERR_BAD_SHAPE
+    assert call(T=2 ** 40, H=2 ** 30) == binding.ASTRA_ERR_BAD_SHAPE
+    assert call(y=Y + 1) == binding.ASTRA_ERR_MISALIGNED
+    assert call(parts=(4 * A, 5 * A + 1)) == binding.ASTRA_ERR_MISALIGNED
+    assert call(parts=(4 * A + 2, 5 * A), dtype=binding.ASTRA_FP32) == binding.ASTRA_ERR_MISALIGNED
+    assert call(y=R) == binding.ASTRA_ERR_OVERLAP                 # y over the residual
+    assert call(parts=(4 * A, Y + 8)) == binding.ASTRA_ERR_OVERLAP    # y over a partial
+    assert call(parts=(R, 5 * A)) == binding.ASTRA_ERR_OVERLAP        # the residual is also a partial
+    assert call(w=Y + 4) == binding.ASTRA_ERR_OVERLAP
+    assert call(T=0) == binding.ASTRA_OK
+    assert call(T=0, parts=None, n=3, y=None, r=None, w=None) == binding.ASTRA_OK
+    import torch
+    if not torch.cuda.is_available():   # well-formed calls reach the launch, which a machine without a GPU refuses
+        assert call(parts=(4 * A, 4 * A)) == binding.ASTRA_ERR_CUDA       # partials may overlap one another
+        assert call(parts=tuple((4 + i) * A for i in range(16)), T=2, H=4100) == binding.ASTRA_ERR_CUDA
+        assert call(parts=(16 * A,), T=1, H=40000, y=32 * A, r=48 * A, w=64 * A) == binding.ASTRA_ERR_CUDA
+
+
 def test_silu_argument_errors(lib):
     f = lib.astra_silu_and_mul
     assert f(None, A, 1, 8, 0, None) == binding.ASTRA_ERR_NULL_POINTER

@@ -66,6 +66,20 @@ def test_operands_on_different_gpus_are_refused_by_the_strided_forms():
                                                fake((2, 3), torch.float32))
 
 
+def test_partials_on_different_gpus_are_accepted_only_as_partials():
+    """The partial hidden states of the all-reduce form are the one operand that may live on other
+    GPUs (that is its purpose); the outputs, the residual and the weight may not."""
+    parts = [fake((4, 64), device=0), fake((4, 64), device=1)]
+    with pytest.raises(ValueError, match="cuda:1"):
+        binding.astra_fused_allreduce_add_rmsnorm(fake((4, 64)), fake((4, 64), device=1), parts, fake((64,)), 1e-6)
+    with pytest.raises(ValueError, match="cuda:1"):
+        binding.astra_fused_allreduce_add_rmsnorm(fake((4, 64)), fake((4, 64)), parts, fake((64,), device=1), 1e-6)
+    with pytest.raises(ValueError):
+        binding.astra_fused_allreduce_add_rmsnorm(fake((4, 64)), fake((4, 64)), [], fake((64,)), 1e-6)
+    with pytest.raises(ValueError):
+        binding.astra_fused_allreduce_add_rmsnorm(fake((4, 64)), fake((4, 64)), [fake((4, 32))], fake((64,)), 1e-6)
+
+
 def test_wrong_dtype_shape_and_layout_are_refused():
     with pytest.raises(TypeError):
         binding.astra_fused_add_rmsnorm(fake((4, 64), torch.int32), fake((4, 64)), fake((64,)), 1e-6)

@@ -1,0 +1,127 @@
+"""GPU parity of astra_fused_allreduce_add_rmsnorm (the all-reduce of the tensor-parallel partial
+hidden states folded into add + RMSNorm) against the oracle, element by element, through the C ABI.
+All partials live on the one GPU here; the kernel reads them with the same plain loads it would use
+for peer-mapped memory.  The residual sum is compared bit for bit, y within the rmsnorm gate."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2509_07506_b200 as astra
+from paper_2509_07506_b200 import workloads as wl
+from parity import check_values
+from test_gpu_parity import NCPU, Guarded, f64, fold, row_chunks
+
+pytestmark = pytest.mark.gpu
+
+BF16, FP16, FP32 = wl.BF16, wl.FP16, wl.FP32
+
+
+def run_allreduce(inp: wl.AllreduceRmsnormInputs, offset=0, prepared=False):
+    T, H = inp.residual.shape
+    gparts = [Guarded(p, offset) for p in inp.parts]
+    gr, gw = Guarded(inp.residual, offset), Guarded(inp.weight, offset)
+    gy = Guarded(torch.zeros_like(inp.residual), offset)
+    if prepared:
+        astra.prepare_fused_allreduce_add_rmsnorm(gy.t, gr.t, [g.t for g in gparts], gw.t, inp.eps)()
+    else:
+        astra.astra_fused_allreduce_add_rmsnorm(gy.t, gr.t, [g.t for g in gparts], gw.t, inp.eps)
+    torch.cuda.synchronize()
+    for g in gparts + [gr, gw, gy]:
+        g.check()
+    for g, p in zip(gparts, inp.parts):
+        assert torch.equal(g.host().view(torch.uint8), p.view(torch.uint8)), "a partial was modified"
+    assert torch.equal(gw.host(), inp.weight)
+    y, r = gy.host(), gr.host()
+    stats = {}
+    for sl in row_chunks(T, H):
+        oy, orr = oracle.fused_allreduce_add_rmsnorm([wl.bits(p[sl]) for p in inp.parts], wl.bits(inp.residual[sl]),
+                                                     wl.bits(inp.weight), inp.eps, inp.dtype, nthreads=NCPU)
+        assert np.array_equal(wl.bits(r[sl]), orr), f"residual sum is not bit-exact in rows {sl.start}..{sl.stop}"
+        fold(stats, check_values(f64(y[sl]), oy, inp.dtype,
+                                 what=f"allreduce rmsnorm {len(inp.parts)} x {(T, H)} rows {sl.start}.."))
+    return stats
+
+
+@pytest.mark.parametrize("n_parts", [2, 4, 8])
+@pytest.mark.parametrize("T,H", [(8192, 4096), (16, 4096), (257, 4100)])
+def test_allreduce_rmsnorm_tensor_parallel_shapes(n_parts, T, H):
+    stats = run_allreduce(wl.allreduce_rmsnorm_inputs(T, H, n_parts, BF16, seed=n_parts))
+    assert stats["max_err_ulp"] <= 2.0
+
+
+@pytest.mark.parametrize("dtype", [BF16, FP16, FP32])
+@pytest.mark.parametrize("n_parts", [1, 2, 3, 5, 8, 16])
+def test_allreduce_rmsnorm_part_counts(dtype, n_parts):
+    run_allreduce(wl.allreduce_rmsnorm_inputs(33, 5120, n_parts, dtype, seed=40 + n_parts))
+
+
+@pytest.mark.parametrize("dtype", [BF16, FP32])
+@pytest.mark.parametrize("n_parts", [2, 5])
+@pytest.mark.parametrize("H", [1, 2, 3, 7, 8, 9, 250, 1000, 4098, 4101, 8192, 11008, 14336, 16384, 16392,
+                               20500, 32768, 40000, 65538])
+def test_allreduce_rmsnorm_widths(dtype, n_parts, H):
+    """Every launch shape: 16-, 8-, 4- and 2-byte vectors, 1 to 8 vectors per thread, two or four
+    partial loads in flight, and the two-sweep kernel for rows too wide for the registers."""
+    run_allreduce(wl.allreduce_rmsnorm_inputs(5 if H < 20000 else 3, H, n_parts, dtype, seed=H))
+
+
+@pytest.mark.parametrize("offset", [1, 2, 4])
+@pytest.mark.parametrize("H", [4096, 4100])
+def test_allreduce_rmsnorm_pointer_offsets(offset, H):
+    run_allreduce(wl.allreduce_rmsnorm_inputs(7, H, 3, BF16, seed=offset), offset=offset)
+
+
+def test_allreduce_rmsnorm_one_part_equals_the_out_of_place_call_bit_for_bit():
+    inp = wl.allreduce_rmsnorm_inputs(300, 4096, 1, BF16, seed=9)
+    x, r, w = inp.parts[0].cuda(), inp.residual.cuda(), inp.weight.cuda()
+    y1, r1 = torch.empty_like(x), r.clone()
+    astra.astra_fused_allreduce_add_rmsnorm(y1, r1, [x], w, inp.eps)
+    y2, r2 = torch.empty_like(x), torch.empty_like(x)
+    astra.astra_fused_add_rmsnorm_ex(y2, r2, x, r, w, inp.eps)
+    assert torch.equal(y1, y2) and torch.equal(r1, r2)
+
+
+def test_allreduce_rmsnorm_depends_on_rank_order_as_the_oracle_does():
+    """Large cancelling partials: the result depends on the order of the additions; the kernel must
+    follow rank order exactly (bit-exact residual for two different orders of the same partials)."""
+    T, H = 9, 4096
+    g = torch.Generator().manual_seed(3)
+    big = (torch.randn((T, H), generator=g) * 1000).to(torch.bfloat16)
+    small = (torch.randn((T, H), generator=g) * 1e-3).to(torch.bfloat16)
+    base = wl.allreduce_rmsnorm_inputs(T, H, 1, BF16, seed=1)
+    for parts in ([big, -big, small], [big, small, -big], [small, big, -big]):
+        run_allreduce(wl.AllreduceRmsnormInputs(parts, base.residual * 1e-3, base.weight, 1e-6, BF16))
+
+
+def test_allreduce_rmsnorm_prepared_and_repeatable():
+    inp = wl.allreduce_rmsnorm_inputs(700, 5120, 4, BF16, seed=77)
+    a = run_allreduce(inp)
+    b = run_allreduce(inp, prepared=True)
+    assert a == b
+    parts = [p.cuda() for p in inp.parts]
+    w = inp.weight.cuda()
+    ref = None
+    for _ in range(6):
+        y, r = torch.empty_like(parts[0]), inp.residual.cuda()
+        astra.astra_fused_allreduce_add_rmsnorm(y, r, parts, w, inp.eps)
+        got = (y.clone(), r.clone())
+        if ref is None:
+            ref = got
+        assert torch.equal(ref[0], got[0]) and torch.equal(ref[1], got[1])
+
+
+def test_allreduce_rmsnorm_binding_refuses_bad_calls():
+    e = lambda *shape: torch.zeros(shape, dtype=torch.bfloat16, device="cuda")  # noqa: E731
+    with pytest.raises(ValueError):
+        astra.astra_fused_allreduce_add_rmsnorm(e(4, 64), e(4, 64), [], e(64), 1e-6)
+    with pytest.raises(ValueError):
+        astra.astra_fused_allreduce_add_rmsnorm(e(4, 64), e(4, 64), [e(4, 64)] * 17, e(64), 1e-6)
+    with pytest.raises(ValueError):
+        astra.astra_fused_allreduce_add_rmsnorm(e(4, 64), e(4, 64), [e(4, 32)], e(64), 1e-6)
+    with pytest.raises(TypeError):
+        astra.astra_fused_allreduce_add_rmsnorm(e(4, 64), e(4, 64), [e(4, 64).float()], e(64), 1e-6)
+    y = e(4, 64)
+    with pytest.raises(astra.AstraError) as err:
+        astra.astra_fused_allreduce_add_rmsnorm(y, e(4, 64), [y, e(4, 64)], e(64), 1e-6)
+    assert err.value.status == 6

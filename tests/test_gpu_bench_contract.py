@@ -35,3 +35,20 @@ def test_bench_prints_one_json_line_with_the_contract_keys():
     e = r["e2e"]
     assert e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0 and 0 < e["value"] < r["value"]
     assert set(r["per_kernel"]) == {"fused_add_rmsnorm", "silu_and_mul", "merge_attn_states_lse"}
+
+
+def test_bench_started_plainly_with_two_ranks_spawns_them():
+    """`python bench.py --gpus 2` without a launcher starts its own two ranks.  With one GPU in the
+    machine the two ranks share it (gloo for the timing reduction; their kernels never wait on one
+    another), which checks the multi-rank host path, not scaling."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--backend", "gloo",
+                          "--steps", "3", "--warmup", "3", "--tokens", "512", "--e2e-steps", "1", "--no-clocks"],
+                         capture_output=True, text=True, timeout=900, cwd=ROOT, env=env)
+    assert out.returncode == 0, out.stderr[-3000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    r = json.loads(lines[0])
+    assert r["n_gpus"] == 2 and r["launcher"] == "self-spawned ranks" and r["scaling"] == "weak"
+    assert "shape_sweep" not in r and "cpu_baseline" not in r   # rank-0-only extras are for the 1-GPU line
+    assert r["value"] > 0 and r["config"]["tokens_per_gpu"] == 512

@@ -346,6 +346,7 @@ def test_empty_batches_through_the_binding():
         s = lambda: torch.empty((0, 4), device="cuda")  # noqa: E731
         astra.astra_merge_attn_states_lse(e(0, 4, 16), s(), e(0, 4, 16), s(), e(0, 4, 16), s())
         astra.astra_merge_attn_states_lse_ex(e(0, 4, 16), None, e(0, 4, 16), s(), e(0, 4, 16), s())
+        astra.astra_fused_allreduce_add_rmsnorm(e(0, 64), e(0, 64), [e(0, 64), e(0, 64)], e(64), 1e-6)
     torch.cuda.synchronize()
 
 
