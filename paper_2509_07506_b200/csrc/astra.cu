@@ -30,6 +30,12 @@ const char kBuildId[] = "astra-build-id:" ASTRA_BUILD_ID;
 // silu_and_mul
 // ---------------------------------------------------------------------------------------------
 // D, the pitches and the pointers are in 16-bit units; UVEC is the vector width in units.
+// Above this many blocks a launch runs long enough that its ramp-up no longer shows, and the extra
+// prefetch requests only cost issue slots (measured: 27 % faster at [128, 14336] and 4 % at
+// [1024, 14336] = 7168 blocks, 2 % slower at [8192, 14336] = 57344 blocks); below it the inputs are
+// requested ahead of the dependency wait.
+constexpr uint32_t kSiluPrefetchMaxBlocks = 1u << 14;
+
 template <int DT, int UVEC, int UNROLL, int THREADS>
 cudaError_t launch_silu(uint16_t *out, const uint16_t *gate, const uint16_t *up, int64_t T, int64_t D,
                         int64_t out_pitch, int64_t gate_pitch, int64_t up_pitch, cudaStream_t stream) {
@@ -42,9 +48,16 @@ cudaError_t launch_silu(uint16_t *out, const uint16_t *gate, const uint16_t *up,
         const uint32_t total = static_cast<uint32_t>(rows * nvec);
         const uint32_t tile = THREADS * UNROLL;
         const uint32_t blocks = (total + tile - 1) / tile;
-        const cudaError_t err = launch(silu_and_mul_kernel<DT, VEC, UNROLL, THREADS>, blocks, THREADS, stream,
-                                       out + t0 * out_pitch, gate + t0 * gate_pitch, up + t0 * up_pitch, total,
-                                       FastDiv::make(static_cast<uint32_t>(nvec)), out_pitch, gate_pitch, up_pitch);
+        const FastDiv per_row = FastDiv::make(static_cast<uint32_t>(nvec));
+        cudaError_t err;
+        if (UVEC == 8 && blocks <= kSiluPrefetchMaxBlocks)
+            err = launch(silu_and_mul_kernel<DT, VEC, UNROLL, THREADS, Ld::StreamReadOnly, St::Stream, THREADS * UNROLL>,
+                         blocks, THREADS, stream, out + t0 * out_pitch, gate + t0 * gate_pitch, up + t0 * up_pitch,
+                         total, per_row, out_pitch, gate_pitch, up_pitch);
+        else
+            err = launch(silu_and_mul_kernel<DT, VEC, UNROLL, THREADS, Ld::StreamReadOnly, St::Stream, 0>, blocks,
+                         THREADS, stream, out + t0 * out_pitch, gate + t0 * gate_pitch, up + t0 * up_pitch, total,
+                         per_row, out_pitch, gate_pitch, up_pitch);
         if (err != cudaSuccess) return err;
     }
   }

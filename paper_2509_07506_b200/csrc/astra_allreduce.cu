@@ -25,16 +25,27 @@ cudaError_t launch_reg(const AllreduceOperands &op, const uint16_t *w, unsigned 
     return cudaErrorInvalidValue;
 }
 
+// Two launch shapes, chosen by the number of rows (measured at H = 4096 with 2, 4 and 8 partials):
+//  - streaming (more rows than one wave of blocks holds): two partial loads in flight per vector
+//    position and 16 units per thread (256-thread blocks at H = 4096).  It beat four and eight in
+//    flight and every other per-thread share by 3 to 25 % at [1024, 4096] and [8192, 4096]: the
+//    registers of a deeper queue cost more occupancy than the queue gains.
+//  - latency (at most one wave: decode-sized batches, where this fusion matters most): up to eight
+//    partial loads in flight and 8 units per thread (512-thread blocks), so that all partials of a
+//    row arrive in one round trip: 2.3 against 3.1 us at [16, 4096] with 8 partials.
+constexpr int kStreamGroup = 2;
+constexpr int kLatencyGroup = 8;
+constexpr int64_t kLatencyRows = 2 * 148;  // two 512-thread blocks per SM on the 148 SMs of a B200
+
 // Per-thread share of a register-resident row for a given width, or 0 if the row does not fit:
-// start at 8 units (one 16-byte vector) when four partials are in flight per vector and at 16
-// otherwise; double it while the block would exceed what the register file allows; halve it while
-// the block would fall under 128 threads.
+// start at `start_units` 16-bit units; double the share while the block would exceed what the
+// register file allows; halve it while the block would fall under 128 threads.
 template <int UVEC, int GROUP>
-inline int pick_vpt(int nvec, int *threads_out) {
+inline int pick_vpt(int nvec, int start_units, int *threads_out) {
     if (UVEC < 4) return 0;  // 2- and 4-byte vectors take the two-sweep kernel
     constexpr int kMaxVpt = 32 / (UVEC < 4 ? 4 : UVEC);
     auto threads_for = [&](int v) { return round_up_to((nvec + v - 1) / v, 32); };
-    int vpt = (GROUP >= 4 ? 8 : 16) / UVEC;
+    int vpt = start_units / UVEC;
     if (vpt < 1) vpt = 1;
     while (vpt <= kMaxVpt && threads_for(vpt) > allreduce_reg_max_threads(UVEC * vpt, GROUP)) vpt <<= 1;
     if (vpt > kMaxVpt) return 0;
@@ -77,21 +88,18 @@ cudaError_t launch_rows(AllreduceOperands op, const uint16_t *w, int64_t T, int 
   return cudaSuccess;
 }
 
-// Four partial loads in flight per vector when there are more than two partials and the row still
-// fits the registers that way; otherwise two.
 template <int DT, int UVEC>
-cudaError_t choose_group(const AllreduceOperands &op, const uint16_t *w, int64_t T, int H, float eps,
+cudaError_t choose_shape(const AllreduceOperands &op, const uint16_t *w, int64_t T, int H, float eps,
                          cudaStream_t stream) {
   if constexpr (UVEC >= Storage<DT>::UNITS) {
     const int nvec = H / (UVEC / Storage<DT>::UNITS);
     int threads = 0;
-    if (op.n_parts > 2) {
-        const int vpt4 = pick_vpt<UVEC, 4>(nvec, &threads);
-        if (vpt4 > 0 || UVEC < 4) return launch_rows<DT, UVEC, 4>(op, w, T, H, eps, vpt4, threads, stream);
+    if (T <= kLatencyRows && op.n_parts > kStreamGroup) {
+        const int vpt = pick_vpt<UVEC, kLatencyGroup>(nvec, 8, &threads);
+        if (vpt > 0) return launch_rows<DT, UVEC, kLatencyGroup>(op, w, T, H, eps, vpt, threads, stream);
     }
-    const int vpt2 = pick_vpt<UVEC, 2>(nvec, &threads);
-    if (vpt2 > 0 || op.n_parts <= 2) return launch_rows<DT, UVEC, 2>(op, w, T, H, eps, vpt2, threads, stream);
-    return launch_rows<DT, UVEC, 4>(op, w, T, H, eps, 0, 0, stream);  // many partials, very wide row
+    const int vpt = pick_vpt<UVEC, kStreamGroup>(nvec, 16, &threads);  // 0: the row does not fit the registers
+    return launch_rows<DT, UVEC, kStreamGroup>(op, w, T, H, eps, vpt, threads, stream);
   }
   return cudaErrorInvalidValue;
 }
@@ -103,10 +111,10 @@ cudaError_t dispatch(const AllreduceOperands &op, const uint16_t *w, int64_t T, 
     pick.extent(static_cast<int64_t>(H) * Storage<DT>::UNITS).pointer(op.r).pointer(op.y).pointer(op.r_out).pointer(w);
     for (int p = 0; p < op.n_parts; ++p) pick.pointer(op.part[p]);
     switch (pick.vec) {
-        case 8: return choose_group<DT, 8>(op, w, T, H, eps, stream);
-        case 4: return choose_group<DT, 4>(op, w, T, H, eps, stream);
-        case 2: return choose_group<DT, 2>(op, w, T, H, eps, stream);
-        default: return choose_group<DT, 1>(op, w, T, H, eps, stream);
+        case 8: return choose_shape<DT, 8>(op, w, T, H, eps, stream);
+        case 4: return choose_shape<DT, 4>(op, w, T, H, eps, stream);
+        case 2: return choose_shape<DT, 2>(op, w, T, H, eps, stream);
+        default: return choose_shape<DT, 1>(op, w, T, H, eps, stream);
     }
 }
 

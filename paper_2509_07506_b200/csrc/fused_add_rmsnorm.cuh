@@ -112,6 +112,11 @@ fused_add_rmsnorm_reg_kernel(RmsnormOperands op, const uint16_t *__restrict__ we
     const uint16_t *rr = op.r + row * op.r_pitch;
     uint16_t *yr = op.y + row * op.y_pitch;
     uint16_t *ror = op.r_out + row * op.r_out_pitch;
+    // the row's two inputs start moving towards L2 while the previous kernel is still draining
+    if (threadIdx.x == 0) {
+        prefetch_l2_range(xr, static_cast<int64_t>(H) * (2 * Storage<DT>::UNITS));
+        prefetch_l2_range(rr, static_cast<int64_t>(H) * (2 * Storage<DT>::UNITS));
+    }
     grid_dependency_wait();
     grid_launch_dependents();
 
@@ -202,6 +207,10 @@ fused_add_rmsnorm_cluster_kernel(RmsnormOperands op, const uint16_t *__restrict_
     uint16_t *yr = op.y + row * op.y_pitch + static_cast<int64_t>(first) * UV;
     uint16_t *ror = op.r_out + row * op.r_out_pitch + static_cast<int64_t>(first) * UV;
     const uint16_t *wr = weight + static_cast<int64_t>(first) * UV;
+    if (threadIdx.x == 0) {
+        prefetch_l2_range(xr, static_cast<int64_t>(count) * UV * 2);
+        prefetch_l2_range(rr, static_cast<int64_t>(count) * UV * 2);
+    }
     grid_dependency_wait();
     grid_launch_dependents();
 

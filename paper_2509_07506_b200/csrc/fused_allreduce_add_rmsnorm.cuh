@@ -12,8 +12,8 @@
 //
 // HBM/NVLink-bound: (N + 3) * 2 bytes per element of 16-bit storage (N partials and r read, y and
 // r_out written).  One block owns a row and keeps the running binary32 sums in registers; the
-// partials are fetched GROUP at a time so that GROUP (+1 for the residual) vector loads per thread
-// are in flight before the first addition.
+// partials are fetched GROUP at a time so that GROUP (+1 for the residual) vector loads per vector
+// position are in flight before the first addition (GROUP = 2 measured best; see the launch code).
 #pragma once
 
 #include "fused_add_rmsnorm.cuh"
@@ -52,7 +52,8 @@ __device__ __forceinline__ void accumulate(float (&s)[VEC], const float (&x)[VEC
 // (one register per element) plus GROUP + 1 packed input copies of it, and the register file is
 // 64 K registers per block.  `units` = 16-bit units of the row per thread.
 __host__ __device__ constexpr int allreduce_reg_max_threads(int units, int group) {
-    return units <= 8 ? 1024 : (units <= 16 ? 512 : (group <= 2 ? 512 : 256));
+    return group > 4 ? (units <= 8 ? 512 : (units <= 16 ? 256 : 128))
+                     : (units <= 8 ? 1024 : (units <= 16 ? 512 : (group <= 2 ? 512 : 256)));
 }
 
 // Register-resident row: thread i owns vectors i, i + blockDim.x, ... (at most VPT of them).
@@ -66,6 +67,9 @@ fused_allreduce_add_rmsnorm_reg_kernel(const __grid_constant__ AllreduceOperands
     const int nvec = H / VEC;
     const int64_t row = static_cast<int64_t>(blockIdx.x) * H * Storage<DT>::UNITS;  // first unit of the row
     const int n = op.n_parts;
+    // The residual row is this GPU's own memory: ask for it ahead of the dependency wait.  The partials
+    // may be another GPU's memory and are left to the ordinary loads below.
+    if (threadIdx.x == 0) prefetch_l2_range(op.r + row, static_cast<int64_t>(H) * (2 * Storage<DT>::UNITS));
     grid_dependency_wait();
     grid_launch_dependents();
 

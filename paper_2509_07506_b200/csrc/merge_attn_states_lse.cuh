@@ -56,7 +56,7 @@ struct MergeStrides {
 };
 
 // Flat indexing over vectors of VEC elements: vector v belongs to row = v / nvec (row = token*Hh+head).
-template <int DT, int VEC, int UNROLL, int THREADS, Ld LDH = Ld::Stream, St STH = St::Stream>
+template <int DT, int VEC, int UNROLL, int THREADS, Ld LDH = Ld::Stream, St STH = St::Stream, bool PREFETCH = true>
 __global__ void __launch_bounds__(THREADS)
 merge_attn_states_lse_kernel(uint16_t *v_out, float *lse_out,
                              const uint16_t *v_a, const float *lse_a,
@@ -64,6 +64,13 @@ merge_attn_states_lse_kernel(uint16_t *v_out, float *lse_out,
                              uint32_t total_vecs, FastDiv nvec) {
     constexpr int UV = VEC * Storage<DT>::UNITS;  // 16-bit units per vector
     const uint32_t base = blockIdx.x * (THREADS * UNROLL) + threadIdx.x;
+    // Ahead of the dependency wait the block asks for its (contiguous) share of both value tensors to
+    // be brought into L2.
+    if (PREFETCH && threadIdx.x == 0 && base < total_vecs) {
+        const uint32_t n = min(static_cast<uint32_t>(THREADS * UNROLL), total_vecs - base);
+        prefetch_l2_range(v_a + static_cast<int64_t>(base) * UV, static_cast<int64_t>(n) * UV * 2);
+        prefetch_l2_range(v_b + static_cast<int64_t>(base) * UV, static_cast<int64_t>(n) * UV * 2);
+    }
     grid_dependency_wait();
     grid_launch_dependents();
     Pack<UV> a[UNROLL], b[UNROLL];

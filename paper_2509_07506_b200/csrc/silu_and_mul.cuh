@@ -49,13 +49,30 @@ __device__ __forceinline__ float2 silu_mul2(float2 a, float2 b) {
 // row = v / nvec, col = v % nvec, nvec = D / VEC.  A block handles THREADS*UNROLL consecutive vectors.
 // gate and up are addressed separately (pointers and row pitches in 16-bit units), which covers both the packed
 // row [a | b] (up = gate + D, equal pitches) and two independent tensors.
-template <int DT, int VEC, int UNROLL, int THREADS, Ld LDH = Ld::StreamReadOnly, St STH = St::Stream>
+template <int DT, int VEC, int UNROLL, int THREADS, Ld LDH = Ld::StreamReadOnly, St STH = St::Stream,
+          int PF_VECS = 0>
 __global__ void __launch_bounds__(THREADS)
 silu_and_mul_kernel(uint16_t *__restrict__ out, const uint16_t *__restrict__ gate,
                     const uint16_t *__restrict__ up, uint32_t total_vecs, FastDiv nvec,
                     int64_t out_pitch, int64_t gate_pitch, int64_t up_pitch) {
     constexpr int UV = VEC * Storage<DT>::UNITS;  // 16-bit units per vector
     const uint32_t base = blockIdx.x * (THREADS * UNROLL) + threadIdx.x;
+    // Ahead of the dependency wait, the block asks for the gate and up bytes of its vectors to be
+    // brought into L2: PF_VECS vectors per request (0 = no prefetch), each request cut at a row end.
+    if constexpr (PF_VECS > 0) {
+        const uint32_t first = blockIdx.x * (THREADS * UNROLL);
+        const uint32_t piece = threadIdx.x * PF_VECS;  // thread t asks for vectors [first + piece, + PF_VECS)
+        if (piece < THREADS * UNROLL && first + piece < total_vecs) {
+            const uint32_t v0 = first + piece;
+            const uint32_t row = nvec.div(v0);
+            const uint32_t col = v0 - row * nvec.d;
+            uint32_t n = min(static_cast<uint32_t>(PF_VECS), total_vecs - v0);
+            n = min(n, nvec.d - col);
+            const int64_t c = static_cast<int64_t>(col) * UV;
+            prefetch_l2_range(gate + (static_cast<int64_t>(row) * gate_pitch + c), static_cast<int64_t>(n) * UV * 2);
+            prefetch_l2_range(up + (static_cast<int64_t>(row) * up_pitch + c), static_cast<int64_t>(n) * UV * 2);
+        }
+    }
     grid_dependency_wait();
     grid_launch_dependents();
     Pack<UV> a[UNROLL], b[UNROLL];

@@ -209,6 +209,27 @@ __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepco
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // ---------------------------------------------------------------------------------------------
+// L2 prefetch of a contiguous byte range with one instruction (the bulk-copy engine's prefetch form;
+// fire and forget: nothing is returned, nothing has to be waited for).  It needs a 16-byte aligned
+// start and a multiple of 16 bytes, so the range is trimmed inward to that; the trimmed edges are
+// simply fetched by the loads later.
+//
+// Use: a block issues it for its inputs BEFORE `grid_dependency_wait()`.  A prefetch consumes no
+// data, and L2 is the point of coherence for everything the previous kernel writes, so this is safe
+// whatever that kernel does to the same addresses; what it buys is that the first-byte latency of
+// this kernel's HBM reads (and, at about one wave of blocks, a good part of the reads themselves)
+// overlaps the previous kernel's drain instead of following it.  Only for memory of this GPU.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void prefetch_l2_range(const void *begin, int64_t bytes) {
+    const uint64_t lo = (reinterpret_cast<uint64_t>(begin) + 15u) & ~static_cast<uint64_t>(15);
+    const uint64_t hi = (reinterpret_cast<uint64_t>(begin) + static_cast<uint64_t>(bytes)) & ~static_cast<uint64_t>(15);
+    if (hi > lo) {
+        const uint32_t n = static_cast<uint32_t>(hi - lo);
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(lo), "r"(n) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Division of a 31-bit index by a launch-constant divisor: q = (n * mul) >> shift, exact for
 // 0 <= n < 2^31 and 1 <= d < 2^31 with shift = 31 + ceil(log2 d), mul = ceil(2^shift / d) <= 2^32 - 1
 // (d = 1 is special-cased so that mul fits 32 bits).
