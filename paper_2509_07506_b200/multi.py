@@ -130,3 +130,18 @@ def row_block_of_rank(total_rows: int, group=None) -> Tuple[int, int]:
     if not (dist.is_available() and dist.is_initialized()):
         return 0, total_rows
     return shard_rows(total_rows, dist.get_world_size(group), dist.get_rank(group))
+
+
+def export_cuda_tensor(t: torch.Tensor):
+    """`export` for exchange_partials when the partial is a CUDA tensor and the ranks are processes of
+    one node: an inter-process memory handle in torch's picklable form.  The tensor must stay alive
+    (and unchanged) for as long as any rank may read it."""
+    from torch.multiprocessing.reductions import reduce_tensor
+    return reduce_tensor(t)
+
+
+def open_cuda_tensor(handle, owner: int) -> torch.Tensor:
+    """`open_remote` for exchange_partials: maps the owner's buffer into this process and returns a
+    tensor over it (no copy).  Reading it is ordinary device memory access through the mapping."""
+    rebuild, args = handle
+    return rebuild(*args)

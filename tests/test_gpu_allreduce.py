@@ -125,3 +125,16 @@ def test_allreduce_rmsnorm_binding_refuses_bad_calls():
     with pytest.raises(astra.AstraError) as err:
         astra.astra_fused_allreduce_add_rmsnorm(y, e(4, 64), [y, e(4, 64)], e(64), 1e-6)
     assert err.value.status == 6
+
+
+def test_allreduce_rmsnorm_reads_partials_of_another_process(tmp_path):
+    """Two ranks as two processes: each holds one partial, maps the other's through an inter-process
+    memory handle, and runs the fused kernel over both; each compares with the oracle.  With one GPU
+    both ranks share it (the kernel never waits on a peer; the ordering is host barriers)."""
+    import os
+    import sys
+    from paper_2509_07506_b200 import multi
+    worker = os.path.join(os.path.dirname(os.path.abspath(__file__)), "tp_worker.py")
+    rc = multi.spawn_ranks([sys.executable, worker, str(tmp_path)], 2, timeout=600)
+    assert rc == 0
+    assert (tmp_path / "tp_gpu_ok0").exists() and (tmp_path / "tp_gpu_ok1").exists()

@@ -386,6 +386,36 @@ def test_prepared_calls_match_plain_calls_bit_for_bit():
     check_values(f64(x2.cpu()), oy, BF16, what="prepared rmsnorm")
 
 
+def test_a_pending_runtime_error_of_the_caller_survives_a_library_call():
+    """An error that some other code left pending in the caller's CUDA runtime (here: a call the
+    runtime refuses on the host, nothing reaches the GPU) must still be there after a successful
+    library call: the library neither reads nor clears the caller's last-error state."""
+    import ctypes
+    try:
+        rt = ctypes.CDLL("libcudart.so.12")   # the runtime torch has loaded
+    except OSError:
+        pytest.skip("the shared CUDA runtime torch uses cannot be opened by name")
+    rt.cudaPeekAtLastError.restype = ctypes.c_int
+    rt.cudaGetLastError.restype = ctypes.c_int
+    rt.cudaSetDevice.restype = ctypes.c_int
+    inp = wl.silu_inputs(8, 1024, BF16, seed=3)
+    d_in = inp.input.cuda()
+    out = torch.empty((8, 1024), dtype=torch.bfloat16, device="cuda")
+    call = astra.prepare_silu_and_mul(out, d_in)
+    torch.cuda.synchronize()
+    assert rt.cudaPeekAtLastError() == 0
+    refused = rt.cudaSetDevice(9999)          # no such device: refused on the host
+    try:
+        assert refused != 0 and rt.cudaPeekAtLastError() == refused
+        call()                                 # a successful launch through the C ABI
+        assert rt.cudaPeekAtLastError() == refused, "the library consumed the caller's pending error"
+    finally:
+        assert rt.cudaGetLastError() == refused    # take it out again
+    assert rt.cudaPeekAtLastError() == 0
+    torch.cuda.synchronize()
+    check_values(f64(out.cpu()), oracle.silu_and_mul(wl.bits(inp.input), BF16), BF16, what="silu after a pending error")
+
+
 def test_binding_rejects_wrong_arguments():
     x = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(TypeError):

@@ -1,0 +1,66 @@
+"""One rank of the two-process check of astra_fused_allreduce_add_rmsnorm with partials that live in
+ANOTHER PROCESS's device memory (mapped through an inter-process handle), started by
+test_gpu_allreduce.py through multi.spawn_ranks.  With one GPU in the machine both ranks use it: the
+kernel has no device-side wait, the ordering is two host barriers, so nothing here depends on the
+two ranks' kernels running at the same time.  Writes <outdir>/tp_gpu_ok<rank> on success."""
+import os
+import sys
+
+import numpy as np
+import torch
+import torch.distributed as dist
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+sys.path.insert(0, os.path.join(ROOT, "tests"))
+
+import oracle  # noqa: E402
+import paper_2509_07506_b200 as astra  # noqa: E402
+from paper_2509_07506_b200 import multi  # noqa: E402
+from paper_2509_07506_b200 import workloads as wl  # noqa: E402
+from parity import check_values  # noqa: E402
+
+
+def main() -> int:
+    out_dir = sys.argv[1]
+    rank, world, local = multi.env_rank_world()
+    dev = torch.device("cuda", local % torch.cuda.device_count())
+    torch.cuda.set_device(dev)
+    multi.init_process_group("gloo")
+    try:
+        T, H = 600, 4096
+        inp = wl.allreduce_rmsnorm_inputs(T, H, world, wl.BF16, seed=11)   # same seed: every rank knows all partials
+        mine = inp.parts[rank].to(dev)
+        r, w = inp.residual.to(dev), inp.weight.to(dev)
+        y = torch.empty_like(mine)
+        torch.cuda.synchronize()
+        parts = multi.exchange_partials(mine, multi.export_cuda_tensor, multi.open_cuda_tensor)
+        assert len(parts) == world and parts[rank] is mine
+        dist.barrier()                      # every partial is written before any rank reads
+        first, count = multi.row_block_of_rank(T)
+        # whole batch (as a tensor-parallel consumer needs it) ...
+        astra.astra_fused_allreduce_add_rmsnorm(y, r, parts, w, inp.eps)
+        # ... and this rank's own row block only (as a sequence-parallel consumer needs it)
+        sl = slice(first, first + count)
+        y2, r2 = torch.empty_like(mine[sl]), inp.residual[sl].to(dev)
+        astra.astra_fused_allreduce_add_rmsnorm(y2, r2, [p[sl] for p in parts], w, inp.eps)
+        torch.cuda.synchronize()
+        dist.barrier()                      # nobody releases its partial while a peer may still read it
+        oy, orr = oracle.fused_allreduce_add_rmsnorm([wl.bits(p) for p in inp.parts], wl.bits(inp.residual),
+                                                     wl.bits(inp.weight), inp.eps, wl.BF16, nthreads=4)
+        assert np.array_equal(wl.bits(r.cpu()), orr), "residual sum is not bit-exact"
+        check_values(y.cpu().to(torch.float64).numpy(), oy, wl.BF16, what=f"rank {rank}: y")
+        assert np.array_equal(wl.bits(r2.cpu()), orr[sl]) and torch.equal(y2, y[sl])
+        for owner in range(world):          # the mapped partials are the owners' bytes
+            assert torch.equal(parts[owner].cpu(), inp.parts[owner])
+        del parts
+        dist.barrier()
+        with open(os.path.join(out_dir, f"tp_gpu_ok{rank}"), "w") as fh:
+            fh.write("ok")
+    finally:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
