@@ -214,28 +214,37 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
     barrier()
     total_ms = c0.elapsed_time(c1)
 
-    # ---- per-kernel timed regions: K back-to-back launches of each kernel on the same buffers -----
-    # (each kernel's working set, 201..705 MB, exceeds L2, so every launch streams from HBM)
+    # ---- per-kernel timed regions: K back-to-back launches of each kernel alone ---------------------
+    # Consecutive launches cycle through independent buffer sets covering eight L2 sizes (four sets for
+    # the rmsnorm, five for the merge, two for silu), so no launch finds any of its own bytes in L2.
+    def copies(keys, nbytes_one):
+        return [{k: (d[k] if i == 0 else d[k].clone()) for k in keys} for i in range(n_cold_sets(nbytes_one))]
+
+    rms_sets = copies(("x", "residual"), nbytes["fused_add_rmsnorm"])
+    silu_sets = copies(("silu_out", "silu_in"), nbytes["silu_and_mul"])
+    merge_sets = copies(("v_out", "lse_out", "v_a", "lse_a", "v_b", "lse_b"), nbytes["merge_attn_states_lse"])
     calls = {
-        "fused_add_rmsnorm": lambda: astra.astra_fused_add_rmsnorm(d["x"], d["residual"], d["weight"], eps),
-        "silu_and_mul": lambda: astra.astra_silu_and_mul(d["silu_out"], d["silu_in"]),
-        "merge_attn_states_lse": lambda: astra.astra_merge_attn_states_lse(
-            d["v_out"], d["lse_out"], d["v_a"], d["lse_a"], d["v_b"], d["lse_b"]),
+        "fused_add_rmsnorm": (rms_sets, lambda b: astra.astra_fused_add_rmsnorm(b["x"], b["residual"], d["weight"], eps)),
+        "silu_and_mul": (silu_sets, lambda b: astra.astra_silu_and_mul(b["silu_out"], b["silu_in"])),
+        "merge_attn_states_lse": (merge_sets, lambda b: astra.astra_merge_attn_states_lse(
+            b["v_out"], b["lse_out"], b["v_a"], b["lse_a"], b["v_b"], b["lse_b"])),
     }
     names = list(calls)
     kernel_ms = {}
     for n in names:
-        fn = calls[n]
-        for _ in range(W):
-            fn()
+        sets, fn = calls[n]
+        for i in range(W):
+            fn(sets[i % len(sets)])
         k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         k0.record()
-        for _ in range(K):
-            fn()
+        for i in range(K):
+            fn(sets[i % len(sets)])
         k1.record()
         torch.cuda.synchronize()
         kernel_ms[n] = k0.elapsed_time(k1) / K
+    per_kernel_sets = {n: len(calls[n][0]) for n in names}
+    del rms_sets, silu_sets, merge_sets, calls
     barrier()
     t_wall1 = time.time()
 
@@ -325,7 +334,8 @@ def run_astra(args, rank: int, world: int, local_rank: int) -> dict | None:
             "parallelism": "rows sharded across GPUs, no collective" if world > 1 else "single GPU",
         },
         "per_kernel": per_kernel,
-        "per_kernel_how": f"each kernel alone: {K} back-to-back launches between two CUDA events, after the chain region",
+        "per_kernel_how": f"each kernel alone: {K} back-to-back launches between two CUDA events, after the chain region, "
+                          f"cycling through {per_kernel_sets} independent buffer sets (the cycle covers eight L2 sizes)",
         "roofline": {"bound": "hbm", "kernel": dominant, "achieved": round(dom_gbs, 1), "peak": peak,
                      "unit": "GB/s", "frac": round(dom_gbs / peak, 4), "traffic": ncu_traffic(dominant, T),
                      "traffic_how": "ncu, per launch: dram__bytes_read.sum + bytes written into L2 by the SMs "
@@ -380,10 +390,25 @@ def _time_launches(fn, reps=100, warmup=20):
     return statistics.median(out)
 
 
+COLD_FOOTPRINT = 8 * L2_BYTES
+
+
+def n_cold_sets(nbytes: int) -> int:
+    """Buffer sets to cycle through so that no launch finds anything of its own in L2: one when a single
+    launch already streams eight L2 sizes, otherwise at least two and enough that the cycle covers
+    eight L2 sizes (at most 64 sets, so the smallest shapes stay partly L2-resident; they are
+    latency-bound either way).  The L2 of this part does not evict in strict LRU order: with a cycle of
+    only 2-3 L2 sizes, lines written 250 MB earlier were still found there ([8192, 4096] in place ran
+    at 36.4 us on one 268 MB set, 40.2 us on two, 40.8 us on four); from a cycle of about 8 L2 sizes on
+    the times stop changing."""
+    if nbytes >= COLD_FOOTPRINT:
+        return 1
+    return max(2, min(64, -(-COLD_FOOTPRINT // max(1, nbytes))))
+
+
 def _rotating(make, nbytes: int):
-    """Enough independent buffer sets that a pass over all of them exceeds twice the L2 size."""
-    n = max(1, min(64, -(-2 * L2_BYTES // max(1, nbytes))))
-    return [make() for _ in range(n)]
+    """Independent buffer sets for L2-cold timing (see n_cold_sets)."""
+    return [make() for _ in range(n_cold_sets(nbytes))]
 
 
 def _time_sets(call, sets):
@@ -430,7 +455,7 @@ def shape_sweep(astra, dev, peak) -> list:
 
     def add(kernel, dtype, shape, nbytes, make, call):
         one = [make()]
-        big = nbytes > 2 * L2_BYTES
+        big = nbytes >= COLD_FOOTPRINT
         many = one if big else _rotating(make, nbytes)
         hot = _time_sets(call, one)
         cold = hot if big else _time_sets(call, many)
@@ -524,7 +549,7 @@ def rmsnorm_cost_model(astra, dev, peak) -> list:
             nbytes = wl.rmsnorm_bytes(T, H)
             make = lambda: (torch.randn((T, H), device=dev).to(td), torch.randn((T, H), device=dev).to(td),  # noqa: E731
                             torch.ones((H,), device=dev, dtype=td))
-            sets = [make()] if nbytes > 2 * L2_BYTES else _rotating(make, nbytes)
+            sets = _rotating(make, nbytes)
             us = _time_graph(lambda b: astra.astra_fused_add_rmsnorm(b[0], b[1], b[2], 1e-5), sets)
             pts.append((T, nbytes, us))
             del sets
@@ -555,8 +580,8 @@ def allreduce_variants(astra, dev, peak) -> list:
             nbytes = wl.allreduce_rmsnorm_bytes(T, H, n)
             make = lambda: ([torch.randn((T, H), device=dev).to(td) for _ in range(n)], torch.randn((T, H), device=dev).to(td),  # noqa: E731
                             torch.empty((T, H), device=dev, dtype=td), torch.ones((H,), device=dev, dtype=td))
-            big = nbytes > 2 * L2_BYTES
-            sets = [make()] if big else _rotating(make, nbytes)
+            big = nbytes > 2 * L2_BYTES   # carries a roofline fraction
+            sets = _rotating(make, nbytes)
             fused = lambda b: astra.astra_fused_allreduce_add_rmsnorm(b[2], b[1], b[0], b[3], 1e-5)  # noqa: E731
 
             def separate(b):
@@ -579,63 +604,63 @@ def allreduce_variants(astra, dev, peak) -> list:
     return rows
 
 
+def _variant_row(name, nbytes, make, call, peak) -> dict:
+    """us/call (paper protocol, through the binding) cycling through L2-cold buffer sets."""
+    sets = _rotating(make, nbytes)
+    us = _time_sets(call, sets)
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return {"call": name, "us_per_call": round(us, 2), "gbs": round(gbs, 1), "buffer_sets": len(sets),
+            **fractions(gbs, peak)}
+
+
 def strided_variants(astra, dev, peak) -> list:
     """The strided / out-of-place entry points at the chain shapes (T = 8192, bf16); each moves the
     same algorithmic bytes as its plain counterpart, so the same roofline applies."""
     T, H, D, Hh, Dh = wl.CHAIN_T, wl.CHAIN_H, wl.CHAIN_D, wl.CHAIN_HEADS, wl.CHAIN_HEAD_DIM
     bf = torch.bfloat16
+    w = torch.ones((H,), device=dev, dtype=bf)
     rows = []
+    rn = lambda *shape: torch.randn(shape, device=dev).to(bf)  # noqa: E731
+    rows.append(_variant_row(
+        "astra_fused_add_rmsnorm_ex out-of-place [8192,4096]", wl.rmsnorm_bytes(T, H),
+        lambda: (torch.empty((T, H), device=dev, dtype=bf), torch.empty((T, H), device=dev, dtype=bf), rn(T, H), rn(T, H)),
+        lambda b: astra.astra_fused_add_rmsnorm_ex(b[0], b[1], b[2], b[3], w, 1e-5), peak))
 
-    def add(name, nbytes, fn):
-        us = _time_launches(fn)
-        gbs = nbytes / (us * 1e-6) / 1e9
-        rows.append({"call": name, "us_per_call": round(us, 2), "gbs": round(gbs, 1), **fractions(gbs, peak)})
-
-    x = torch.randn((T, H), device=dev).to(bf); r = torch.randn((T, H), device=dev).to(bf)
-    y = torch.empty_like(x); ro = torch.empty_like(x); w = torch.ones((H,), device=dev, dtype=bf)
-    add("astra_fused_add_rmsnorm_ex out-of-place [8192,4096]", wl.rmsnorm_bytes(T, H),
-        lambda: astra.astra_fused_add_rmsnorm_ex(y, ro, x, r, w, 1e-5))
-    wide = torch.randn((T, 2 * H + 256), device=dev).to(bf)
-    xs, rs = wide[:, :H], wide[:, H + 128:2 * H + 128]
-    add("astra_fused_add_rmsnorm_ex in place on slices of a [8192, 8448] buffer", wl.rmsnorm_bytes(T, H),
-        lambda: astra.astra_fused_add_rmsnorm_ex(xs, rs, xs, rs, w, 1e-5))
-    del x, r, y, ro, wide
-    gate = torch.randn((T, D), device=dev).to(bf); up = torch.randn((T, D), device=dev).to(bf)
-    out = torch.empty((T, D), device=dev, dtype=bf)
-    add("astra_silu_and_mul_ex separate gate and up tensors [8192,14336]", wl.silu_bytes(T, D),
-        lambda: astra.astra_silu_and_mul_ex(out, gate, up))
-    del gate, up, out
-    va = torch.randn((T, Hh, Dh), device=dev).to(bf); vb = torch.randn((T, Hh, Dh), device=dev).to(bf)
-    vo = torch.empty_like(va)
-    sa = (torch.rand((Hh, T), device=dev) * 30 - 10).t(); sb = (torch.rand((Hh, T), device=dev) * 30 - 10).t()
-    so = torch.empty((Hh, T), device=dev).t()
-    add("astra_merge_attn_states_lse_ex head-major scores [8192,32,128]", wl.merge_bytes(T, Hh, Dh),
-        lambda: astra.astra_merge_attn_states_lse_ex(vo, so, va, sa, vb, sb))
+    def slices():
+        wide = rn(T, 2 * H + 256)
+        return wide[:, :H], wide[:, H + 128:2 * H + 128]
+    rows.append(_variant_row(
+        "astra_fused_add_rmsnorm_ex in place on slices of a [8192, 8448] buffer", wl.rmsnorm_bytes(T, H), slices,
+        lambda b: astra.astra_fused_add_rmsnorm_ex(b[0], b[1], b[0], b[1], w, 1e-5), peak))
+    rows.append(_variant_row(
+        "astra_silu_and_mul_ex separate gate and up tensors [8192,14336]", wl.silu_bytes(T, D),
+        lambda: (torch.empty((T, D), device=dev, dtype=bf), rn(T, D), rn(T, D)),
+        lambda b: astra.astra_silu_and_mul_ex(b[0], b[1], b[2]), peak))
+    rows.append(_variant_row(
+        "astra_merge_attn_states_lse_ex head-major scores [8192,32,128]", wl.merge_bytes(T, Hh, Dh),
+        lambda: (torch.empty((T, Hh, Dh), device=dev, dtype=bf), torch.empty((Hh, T), device=dev).t(), rn(T, Hh, Dh),
+                 (torch.rand((Hh, T), device=dev) * 30 - 10).t(), rn(T, Hh, Dh), (torch.rand((Hh, T), device=dev) * 30 - 10).t()),
+        lambda b: astra.astra_merge_attn_states_lse_ex(b[0], b[1], b[2], b[3], b[4], b[5]), peak))
     return rows
 
 
 def fp32_variants(astra, dev, peak) -> list:
     """The three operations on fp32 storage at the chain shapes (twice the bytes of the bf16 calls)."""
     T, H, D, Hh, Dh = wl.CHAIN_T, wl.CHAIN_H, wl.CHAIN_D, wl.CHAIN_HEADS, wl.CHAIN_HEAD_DIM
-    rows = []
-
-    def add(name, nbytes, fn):
-        us = _time_launches(fn)
-        gbs = nbytes / (us * 1e-6) / 1e9
-        rows.append({"call": name, "us_per_call": round(us, 2), "gbs": round(gbs, 1), **fractions(gbs, peak)})
-
-    x = torch.randn((T, H), device=dev); r = torch.randn((T, H), device=dev); w = torch.ones((H,), device=dev)
-    add("astra_fused_add_rmsnorm fp32 [8192,4096]", wl.rmsnorm_bytes(T, H, 4),
-        lambda: astra.astra_fused_add_rmsnorm(x, r, w, 1e-5))
-    del x, r, w
-    si = torch.randn((T, 2 * D), device=dev); so = torch.empty((T, D), device=dev)
-    add("astra_silu_and_mul fp32 [8192,2*14336]", wl.silu_bytes(T, D, 4), lambda: astra.astra_silu_and_mul(so, si))
-    del si, so
-    va = torch.randn((T, Hh, Dh), device=dev); vb = torch.randn((T, Hh, Dh), device=dev); vo = torch.empty_like(va)
-    sa = torch.rand((T, Hh), device=dev) * 30 - 10; sb = torch.rand((T, Hh), device=dev) * 30 - 10
-    lo = torch.empty_like(sa)
-    add("astra_merge_attn_states_lse fp32 [8192,32,128]", wl.merge_bytes(T, Hh, Dh, 4),
-        lambda: astra.astra_merge_attn_states_lse(vo, lo, va, sa, vb, sb))
+    w = torch.ones((H,), device=dev)
+    rn = lambda *shape: torch.randn(shape, device=dev)  # noqa: E731
+    rows = [
+        _variant_row("astra_fused_add_rmsnorm fp32 [8192,4096]", wl.rmsnorm_bytes(T, H, 4),
+                     lambda: (rn(T, H), rn(T, H)),
+                     lambda b: astra.astra_fused_add_rmsnorm(b[0], b[1], w, 1e-5), peak),
+        _variant_row("astra_silu_and_mul fp32 [8192,2*14336]", wl.silu_bytes(T, D, 4),
+                     lambda: (torch.empty((T, D), device=dev), rn(T, 2 * D)),
+                     lambda b: astra.astra_silu_and_mul(b[0], b[1]), peak),
+        _variant_row("astra_merge_attn_states_lse fp32 [8192,32,128]", wl.merge_bytes(T, Hh, Dh, 4),
+                     lambda: (torch.empty((T, Hh, Dh), device=dev), torch.empty((T, Hh), device=dev), rn(T, Hh, Dh),
+                              torch.rand((T, Hh), device=dev) * 30 - 10, rn(T, Hh, Dh), torch.rand((T, Hh), device=dev) * 30 - 10),
+                     lambda b: astra.astra_merge_attn_states_lse(b[0], b[1], b[2], b[3], b[4], b[5]), peak),
+    ]
     return rows
 
 

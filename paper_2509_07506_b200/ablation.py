@@ -130,9 +130,10 @@ def _graph_us(call, sets, launches=100) -> float:
 
 
 def _sets(make, nbytes):
-    n = max(1, min(64, -(-2 * L2_BYTES // max(1, nbytes))))
-    if nbytes > 2 * L2_BYTES:
-        n = 1
+    """Independent buffer sets to cycle through so that no launch finds its own bytes in L2: one if a
+    single launch streams eight L2 sizes, otherwise at least two and enough to cover eight L2 sizes
+    (this part's L2 keeps lines far longer than strict LRU eviction would)."""
+    n = 1 if nbytes >= 8 * L2_BYTES else max(2, min(64, -(-8 * L2_BYTES // max(1, nbytes))))
     return [make() for _ in range(n)]
 
 

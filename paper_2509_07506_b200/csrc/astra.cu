@@ -31,9 +31,9 @@ const char kBuildId[] = "astra-build-id:" ASTRA_BUILD_ID;
 // ---------------------------------------------------------------------------------------------
 // D, the pitches and the pointers are in 16-bit units; UVEC is the vector width in units.
 // Above this many blocks a launch runs long enough that its ramp-up no longer shows, and the extra
-// prefetch requests only cost issue slots (measured: 27 % faster at [128, 14336] and 4 % at
-// [1024, 14336] = 7168 blocks, 2 % slower at [8192, 14336] = 57344 blocks); below it the inputs are
-// requested ahead of the dependency wait.
+// prefetch requests only cost issue slots (measured, L2-cold: 24 % faster at [128, 14336], 5 % at
+// [1024, 14336] = 7168 blocks, 0.5 % at [4096, 14336], 1.6 % slower at [8192, 14336] = 57344 blocks);
+// below it the inputs are requested ahead of the dependency wait.
 constexpr uint32_t kSiluPrefetchMaxBlocks = 1u << 14;
 
 template <int DT, int UVEC, int UNROLL, int THREADS>
