@@ -32,7 +32,8 @@ cudaError_t launch_reg(const AllreduceOperands &op, const uint16_t *w, unsigned 
 //    registers of a deeper queue cost more occupancy than the queue gains.
 //  - latency (at most one wave: decode-sized batches, where this fusion matters most): up to eight
 //    partial loads in flight and 8 units per thread (512-thread blocks), so that all partials of a
-//    row arrive in one round trip: 2.3 against 3.1 us at [16, 4096] with 8 partials.
+//    row arrive in one round trip: 2.5 against 3.9 us at [16, 4096] with 8 partials (with one or two
+//    partials the queue stays at two, the per-thread share is still 8 units: 1.8 against 2.0 us).
 constexpr int kStreamGroup = 2;
 constexpr int kLatencyGroup = 8;
 constexpr int64_t kLatencyRows = 2 * 148;  // two 512-thread blocks per SM on the 148 SMs of a B200
@@ -98,7 +99,8 @@ cudaError_t choose_shape(const AllreduceOperands &op, const uint16_t *w, int64_t
         const int vpt = pick_vpt<UVEC, kLatencyGroup>(nvec, 8, &threads);
         if (vpt > 0) return launch_rows<DT, UVEC, kLatencyGroup>(op, w, T, H, eps, vpt, threads, stream);
     }
-    const int vpt = pick_vpt<UVEC, kStreamGroup>(nvec, 16, &threads);  // 0: the row does not fit the registers
+    const int start_units = T <= kLatencyRows ? 8 : 16;
+    const int vpt = pick_vpt<UVEC, kStreamGroup>(nvec, start_units, &threads);  // 0: the row does not fit the registers
     return launch_rows<DT, UVEC, kStreamGroup>(op, w, T, H, eps, vpt, threads, stream);
   }
   return cudaErrorInvalidValue;
