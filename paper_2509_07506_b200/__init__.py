@@ -4,6 +4,7 @@
 seeded synthetic inputs; ``build`` compiles the shared library.  Importing the package does not
 load the library; the first call does, and fails loudly if it has not been built.
 """
+from .graphs import CapturedCalls  # noqa: F401
 from .binding import (  # noqa: F401
     AstraError,
     PreparedCall,

@@ -386,6 +386,45 @@ def test_prepared_calls_match_plain_calls_bit_for_bit():
     check_values(f64(x2.cpu()), oy, BF16, what="prepared rmsnorm")
 
 
+def test_decode_chain_replayed_from_a_graph_matches_the_oracle():
+    """The three calls at a decode-sized batch, captured once and replayed with new inputs: every
+    replay's outputs are compared with the oracle (and are bit-identical to the eager calls')."""
+    T, H, D, Hh, Dh = 16, 4096, 14336, 32, 128
+    dev = "cuda"
+    x = torch.empty((T, H), dtype=torch.bfloat16, device=dev); r = torch.empty_like(x)
+    w = torch.empty((H,), dtype=torch.bfloat16, device=dev)
+    si = torch.empty((T, 2 * D), dtype=torch.bfloat16, device=dev); so = torch.empty((T, D), dtype=torch.bfloat16, device=dev)
+    va = torch.empty((T, Hh, Dh), dtype=torch.bfloat16, device=dev); vb = torch.empty_like(va); vo = torch.empty_like(va)
+    sa = torch.empty((T, Hh), device=dev); sb = torch.empty_like(sa); lo = torch.empty_like(sa)
+    chain = astra.CapturedCalls([astra.prepare_fused_add_rmsnorm(x, r, w, 1e-5), astra.prepare_silu_and_mul(so, si),
+                                 astra.prepare_merge_attn_states_lse(vo, lo, va, sa, vb, sb)])
+    for seed in (101, 102, 103):
+        rms = wl.rmsnorm_inputs(T, H, BF16, eps=1e-5, seed=seed)
+        sil = wl.silu_inputs(T, D, BF16, seed=seed)
+        mer = wl.merge_inputs(T, Hh, Dh, BF16, seed=seed, neg_inf_frac=0.05)
+        x.copy_(rms.x); r.copy_(rms.residual); w.copy_(rms.weight); si.copy_(sil.input)
+        va.copy_(mer.v_a); vb.copy_(mer.v_b); sa.copy_(mer.lse_a); sb.copy_(mer.lse_b)
+        so.zero_(); vo.zero_(); lo.zero_()
+        chain.replay()
+        torch.cuda.synchronize()
+        oy, orr = oracle.fused_add_rmsnorm(wl.bits(rms.x), wl.bits(rms.residual), wl.bits(rms.weight), 1e-5, BF16)
+        assert np.array_equal(wl.bits(r.cpu()), orr)
+        check_values(f64(x.cpu()), oy, BF16, what="graph replay: rmsnorm")
+        check_values(f64(so.cpu()), oracle.silu_and_mul(wl.bits(sil.input), BF16), BF16, what="graph replay: silu")
+        ov, ol = oracle.merge_attn_states_lse(wl.bits(mer.v_a), mer.lse_a.numpy(), wl.bits(mer.v_b), mer.lse_b.numpy(), BF16)
+        check_values(f64(vo.cpu()), ov, BF16, extra=merge_floor(f64(mer.v_a), mer.lse_a.numpy(), f64(mer.v_b), mer.lse_b.numpy(), BF16),
+                     what="graph replay: merge")
+        check_lse(lo.cpu().numpy(), ol, what="graph replay: merge lse")
+        # the same inputs through eager calls: identical bits
+        x2, r2 = rms.x.cuda(), rms.residual.cuda()
+        so2, vo2, lo2 = torch.empty_like(so), torch.empty_like(vo), torch.empty_like(lo)
+        astra.astra_fused_add_rmsnorm(x2, r2, w, 1e-5)
+        astra.astra_silu_and_mul(so2, si)
+        astra.astra_merge_attn_states_lse(vo2, lo2, va, sa, vb, sb)
+        assert torch.equal(x, x2) and torch.equal(r, r2) and torch.equal(so, so2) and torch.equal(vo, vo2)
+        assert torch.equal(lo.view(torch.int32), lo2.view(torch.int32))
+
+
 def test_a_pending_runtime_error_of_the_caller_survives_a_library_call():
     """An error that some other code left pending in the caller's CUDA runtime (here: a call the
     runtime refuses on the host, nothing reaches the GPU) must still be there after a successful
