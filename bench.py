@@ -41,7 +41,7 @@ NOMINAL_HBM_GBS = 7700.0   # HGX B200 data-sheet figure
 HBM3E_SPEC_GBS = 8000.0    # 3996 MHz x 2 x 8192 bit: the interface's own ceiling
 FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 * 1024 * 1024
-TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_traffic_T4096.json")
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_traffic_T4096.txt")
 
 
 def ncu_traffic(kernel: str, tokens: int):
