@@ -449,8 +449,9 @@ def _time_graph(call, sets, launches=100):
 def shape_sweep(astra, dev, peak) -> list:
     """us/call for configs[0..2] and every point of the fused_add_rmsnorm sweep (configs[3]).
     `us_hot` repeats one buffer set (it stays in L2 when it fits); `us_cold` cycles through enough
-    sets to defeat L2; `*_graph` are the same launches replayed from a CUDA graph (device time only).  Shapes whose working set exceeds L2 give the same number both ways and carry
-    the roofline fraction; the small ones are launch-latency bound and are reported in us only."""
+    sets to defeat L2 (n_cold_sets); `*_graph` are the same launches replayed from a CUDA graph (device
+    time only).  Shapes that stream more than two L2 sizes carry the roofline fraction of their L2-cold
+    time; the small ones are launch-latency bound and are reported in us only."""
     rows = []
 
     def add(kernel, dtype, shape, nbytes, make, call):
@@ -467,7 +468,7 @@ def shape_sweep(astra, dev, peak) -> list:
         best = cold if big else row["us_cold_graph"]
         gbs = nbytes / (best * 1e-6) / 1e9
         row["gbs_cold"] = round(gbs, 1)
-        if big:
+        if nbytes > 2 * L2_BYTES:      # streaming sizes carry the roofline fraction (of the L2-cold time)
             row.update(fractions(gbs, peak))
         else:
             row["frac_of_measured_peak"] = None

@@ -294,6 +294,76 @@ def test_interleaved_slices_of_one_buffer_are_not_overlap(lib):
     assert r  # the accepting direction is covered by the GPU tests (slices of one buffer)
 
 
+def test_overlap_check_against_brute_force(lib):
+    """The pitched overlap test that guards the out-of-place / sliced calls, against element sets
+    enumerated by brute force: with equal pitches it must be exact (slices of one buffer interleave
+    without sharing an element), with different pitches it may only err towards reporting overlap.
+    Runs where no GPU exists: a call that passes the check goes on to the launch, which such a
+    machine refuses (ASTRA_ERR_CUDA), so nothing is ever launched on these fake addresses."""
+    import random
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a CUDA device is present; the fake addresses of this test must not be launched on")
+    f = lib.astra_fused_add_rmsnorm_ex
+    rng = random.Random(7)
+    base, far = 64 * A, 4096 * A
+    checked = {"overlap": 0, "clear": 0}
+    for _ in range(4000):
+        T, H = rng.randint(1, 5), rng.randint(1, 6)
+        px, py = rng.randint(H, 12), rng.randint(H, 12)
+        if rng.random() < 0.6:
+            py = px
+        dy = rng.randint(-40, 40)                      # y starts dy elements after x
+        x, y = base, base + 2 * dy
+        ex = {2 * (t * px + j) for t in range(T) for j in range(H)}
+        ey = {2 * (dy + t * py + j) for t in range(T) for j in range(H)}
+        same = (dy == 0 and px == py)
+        truly = bool(ex & ey) and not same
+        st = f(y, far, x, 2 * far, 3 * far, T, H, py, H, px, H, 1e-6, 0, None)
+        assert st in (binding.ASTRA_ERR_OVERLAP, binding.ASTRA_ERR_CUDA)
+        reported = st == binding.ASTRA_ERR_OVERLAP
+        if px == py or T == 1:
+            assert reported == truly, (T, H, px, py, dy)
+        else:
+            assert reported or not truly, (T, H, px, py, dy)   # never a missed overlap
+        checked["overlap" if truly else "clear"] += 1
+    assert checked["overlap"] > 300 and checked["clear"] > 300
+
+
+def test_strided_output_rows_never_share_elements(lib):
+    """The strided merge writes one row of D elements per (token, head); a stride pair under which
+    two of those rows share an element must be refused (ASTRA_ERR_BAD_SHAPE), checked against brute
+    force.  The test may refuse some exotic disjoint layouts, never accept an overlapping one.
+    Runs only where no GPU exists (accepted calls end at the refused launch)."""
+    import ctypes as C
+    import random
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a CUDA device is present; the fake addresses of this test must not be launched on")
+    f = lib.astra_merge_attn_states_lse_ex
+    rng = random.Random(11)
+    far = 4096 * A
+    accepted = refused_disjoint = refused_overlapping = 0
+    for _ in range(4000):
+        T, Hh, D = rng.randint(1, 4), rng.randint(1, 4), rng.randint(1, 5)
+        st, sh = rng.randint(0, 24), rng.randint(0, 24)
+        rows = [set(range(t * st + h * sh, t * st + h * sh + D)) for t in range(T) for h in range(Hh)]
+        overlapping = any(rows[i] & rows[j] for i in range(len(rows)) for j in range(i))
+        big = 64    # input and score strides: dense in a space of their own
+        strides = (C.c_int64 * 12)(big * 4, big, big * 4, big, st, sh, Hh, 1, Hh, 1, Hh, 1)
+        code = f(far, 2 * far, 3 * far, 4 * far, 5 * far, 6 * far, T, Hh, D, strides, 0, None)
+        assert code in (binding.ASTRA_ERR_BAD_SHAPE, binding.ASTRA_ERR_CUDA), code
+        if code == binding.ASTRA_ERR_CUDA:
+            assert not overlapping, (T, Hh, D, st, sh)   # an accepted layout is always disjoint
+            accepted += 1
+        elif overlapping:
+            refused_overlapping += 1
+        else:
+            refused_disjoint += 1
+    assert accepted > 300 and refused_overlapping > 300
+    assert refused_disjoint < accepted   # the check is conservative only for unusual interleavings
+
+
 def test_fp32_storage_needs_four_byte_alignment(lib):
     FP32 = binding.ASTRA_FP32
     assert FP32 == 2
