@@ -57,9 +57,19 @@ __host__ __device__ constexpr int allreduce_reg_max_threads(int units, int group
 }
 
 // Register-resident row: thread i owns vectors i, i + blockDim.x, ... (at most VPT of them).
-// Requires nvec = H / VEC <= VPT * blockDim.x and blockDim.x <= allreduce_reg_max_threads(...).
-template <int DT, int VEC, int VPT, int GROUP>
-__global__ void __launch_bounds__(allreduce_reg_max_threads(VEC * VPT * Storage<DT>::UNITS, GROUP))
+// Requires nvec = H / VEC <= VPT * blockDim.x and blockDim.x <= allreduce_reg_max_threads(...), or
+// blockDim.x <= kAllreduceDenseThreads for the DENSE instantiation: blocks of at most 256 threads
+// whose register allocation is held to 48 so that five of them are resident per SM instead of four
+// (for two loads in flight and 16 units per thread that costs no spill).  Measured at [8192, 4096],
+// L2-cold: 50.8 -> 50.5 us with 2 partials, 71.5 -> 70.4 us with 4, 112.2 -> 110.3 us with 8; at
+// [1024, 4096] it is neutral or slower (16.1 -> 16.5 us with 8 partials), so the launch code uses it
+// for long streams only.
+constexpr int kAllreduceDenseThreads = 256;
+constexpr int kAllreduceDenseBlocks = 5;
+
+template <int DT, int VEC, int VPT, int GROUP, bool DENSE = false>
+__global__ void __launch_bounds__(DENSE ? kAllreduceDenseThreads : allreduce_reg_max_threads(VEC * VPT * Storage<DT>::UNITS, GROUP),
+                                  DENSE ? kAllreduceDenseBlocks : 1)
 fused_allreduce_add_rmsnorm_reg_kernel(const __grid_constant__ AllreduceOperands op,
                                        const uint16_t *__restrict__ weight, int H, float eps, float inv_H) {
     constexpr int UV = VEC * Storage<DT>::UNITS;  // 16-bit units per vector
@@ -81,8 +91,15 @@ fused_allreduce_add_rmsnorm_reg_kernel(const __grid_constant__ AllreduceOperands
         if (v < nvec) pr[i] = load<UV, Ld::Stream>(op.r + row + v * UV);
     }
 
+    // The loop over groups is unrolled to the largest supported count and left by a break: every copy
+    // then has a constant p0 (the first one initialises the sums without a test) and the compiler may
+    // move a group's loads above the additions of the group before it.  Measured against the rolled
+    // loop at [8192, 4096], L2-cold: 54.1 -> 50.8 us with 2 partials, 74.5 -> 71.8 us with 4,
+    // 113.8 -> 111.8 us with 8.
     float s[VPT][VEC];
-    for (int p0 = 0; p0 < n; p0 += GROUP) {
+#pragma unroll
+    for (int p0 = 0; p0 < kMaxParts; p0 += GROUP) {
+        if (p0 >= n) break;
         Pack<UV> px[GROUP][VPT];
 #pragma unroll
         for (int g = 0; g < GROUP; ++g) {
@@ -156,7 +173,9 @@ __device__ __forceinline__ void rank_order_sum(const AllreduceOperands &op, int6
     constexpr int UV = VEC * Storage<DT>::UNITS;
     const int n = op.n_parts;
     const Pack<UV> pr = load<UV, Ld::Stream>(op.r + at);
-    for (int p0 = 0; p0 < n; p0 += GROUP) {
+#pragma unroll
+    for (int p0 = 0; p0 < kMaxParts; p0 += GROUP) {  // unrolled and left by a break, as in the kernel above
+        if (p0 >= n) break;
         Pack<UV> px[GROUP];
 #pragma unroll
         for (int g = 0; g < GROUP; ++g)

@@ -50,6 +50,13 @@ def test_allreduce_rmsnorm_tensor_parallel_shapes(n_parts, T, H):
     assert stats["max_err_ulp"] <= 2.0
 
 
+@pytest.mark.parametrize("dtype,H", [(FP16, 4096), (FP32, 2048), (BF16, 2048), (FP32, 1024)])
+def test_allreduce_rmsnorm_long_streams(dtype, H):
+    """From 4096 rows on, rows of 16-byte vectors with 16 units per thread take the register-capped
+    instantiation of the kernel: every storage type of it, every row, against the oracle."""
+    run_allreduce(wl.allreduce_rmsnorm_inputs(4096 + 5, H, 3, dtype, seed=H + 1))
+
+
 @pytest.mark.parametrize("dtype", [BF16, FP16, FP32])
 @pytest.mark.parametrize("n_parts", [1, 2, 3, 5, 8, 16])
 def test_allreduce_rmsnorm_part_counts(dtype, n_parts):
