@@ -15,6 +15,7 @@ from typing import Optional
 import torch
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libastra.so")
+FASTCALL_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "_astra_fastcall.so")
 
 ASTRA_BF16 = 0
 ASTRA_FP16 = 1
@@ -83,8 +84,35 @@ def load_library() -> ctypes.CDLL:
     lib.astra_build_id.argtypes = []
     lib.astra_build_id.restype = ctypes.c_char_p
     _refuse_stale(lib)
+    _load_fastcall(lib)
     _lib = lib
     return lib
+
+
+_fast = None  # the _astra_fastcall extension module, once loaded
+
+
+def _load_fastcall(lib) -> None:
+    """Import the `_astra_fastcall` extension from the package directory and give it the addresses of
+    the entry points resolved above.  It re-issues prepared calls without going through ctypes (about
+    1 us less host time per launch) and, like the library, it is required: a missing or stale module
+    is an error, not a reason to take another route."""
+    global _fast
+    try:
+        from . import _astra_fastcall as fast
+    except ImportError as exc:
+        raise ImportError(
+            f"{FASTCALL_PATH} is missing or cannot be loaded ({exc}): build it with "
+            "`python -m paper_2509_07506_b200.build`") from exc
+    from . import build as _build
+    if os.path.isdir(_build.CSRC) and os.path.isdir(_build.INCLUDE) and fast.build_id() != _build.source_hash():
+        raise ImportError(f"{FASTCALL_PATH} was built from other sources: rebuild it with "
+                          "`python -m paper_2509_07506_b200.build`")
+    for kind, fn in ((fast.KIND_RMSNORM, lib.astra_fused_add_rmsnorm), (fast.KIND_SILU, lib.astra_silu_and_mul),
+                     (fast.KIND_MERGE, lib.astra_merge_attn_states_lse),
+                     (fast.KIND_ALLREDUCE_RMSNORM, lib.astra_fused_allreduce_add_rmsnorm)):
+        fast.bind(kind, ctypes.cast(fn, ctypes.c_void_p).value)
+    _fast = fast
 
 
 def _refuse_stale(lib) -> None:
@@ -169,21 +197,25 @@ class PreparedCall:
 
     The plain functions below check every tensor, read its address and convert the arguments on
     each call; for the small shapes of decode steps that host work takes longer than the kernel.
-    A prepared call does all of it once: it keeps the library function and the converted argument
-    tuple (and references to the tensors, so their addresses stay valid) and ``__call__`` only looks
-    up the current stream and issues the launch.  The tensors' contents may change between calls;
-    their addresses, shapes and dtypes are fixed at preparation.  Results are identical to the plain
-    call's, which is itself ``prepare(...)()``.
+    A prepared call does all of it once: it keeps the converted arguments in a C struct of the
+    ``_astra_fastcall`` extension (and references to the tensors, so their addresses stay valid) and
+    ``__call__`` only looks up the current stream and hands the struct to the entry point, without
+    ctypes in between.  The C entry point still checks every argument on every launch.  The tensors'
+    contents may change between calls; their addresses, shapes and dtypes are fixed at preparation.
+    Results are identical to the plain call's, which is itself ``prepare(...)()``.
+    ``via_ctypes()`` issues the same call through ctypes (kept to compare the two routes).
     """
 
-    __slots__ = ("name", "_fn", "_args", "_device", "_keep")
+    __slots__ = ("name", "_fn", "_make_args", "_device", "_keep", "_ready", "_launch")
 
-    def __init__(self, name: str, fn, args: tuple, device: torch.device, keep: tuple):
+    def __init__(self, name: str, fn, make_args, device: torch.device, keep: tuple, ready):
         self.name = name
         self._fn = fn
-        self._args = args
+        self._make_args = make_args  # builds the ctypes argument tuple, only when via_ctypes() asks for it
         self._device = device.index if device.index is not None else torch.cuda.current_device()
         self._keep = keep
+        self._ready = ready
+        self._launch = _fast.launch
 
     def __call__(self, stream: Optional[torch.cuda.Stream] = None) -> None:
         dev = self._device
@@ -194,12 +226,27 @@ class PreparedCall:
         else:
             handle = torch.cuda.current_stream(dev).cuda_stream
         if _raw_current_device() == dev:
-            st = self._fn(*self._args, handle)
+            st = self._launch(self._ready, handle)
         else:  # the C side launches on the current device
             with torch.cuda.device(dev):
-                st = self._fn(*self._args, handle)
+                st = self._launch(self._ready, handle)
         if st != ASTRA_OK:
             raise AstraError(st, self.name)
+
+    def via_ctypes(self, stream: Optional[torch.cuda.Stream] = None) -> None:
+        """The same launch issued through ctypes instead of the extension module."""
+        handle = stream.cuda_stream if stream is not None else _stream_of(self._device)
+        args = self._make_args()
+        with torch.cuda.device(self._device):
+            st = self._fn(*args, handle)
+        if st != ASTRA_OK:
+            raise AstraError(st, self.name)
+
+
+def _stream_of(dev: int) -> int:
+    if _raw_current_stream is not None:
+        return _raw_current_stream(dev)
+    return torch.cuda.current_stream(dev).cuda_stream
 
 
 _raw_current_device = getattr(torch._C, "_cuda_getDevice", None) or torch.cuda.current_device
@@ -219,10 +266,13 @@ def prepare_fused_add_rmsnorm(x: torch.Tensor, residual: torch.Tensor, weight: t
     T, H = x.shape
     _check(residual, "residual", x.dtype, (T, H), x.device)
     _check(weight, "weight", x.dtype, (H,), x.device)
-    args = (_ptr(x), _ptr(residual), _ptr(weight), ctypes.c_int64(T), ctypes.c_int64(H),
-            ctypes.c_float(float(eps)), ctypes.c_int(code))
-    return PreparedCall("astra_fused_add_rmsnorm", load_library().astra_fused_add_rmsnorm, args, x.device,
-                        (x, residual, weight))
+    args = lambda: (_ptr(x), _ptr(residual), _ptr(weight), ctypes.c_int64(T), ctypes.c_int64(H),  # noqa: E731
+                    ctypes.c_float(float(eps)), ctypes.c_int(code))
+    lib = load_library()
+    ready = _fast.prepare(_fast.KIND_RMSNORM, (x.data_ptr(), residual.data_ptr(), weight.data_ptr()), (T, H),
+                          float(eps), code, ())
+    return PreparedCall("astra_fused_add_rmsnorm", lib.astra_fused_add_rmsnorm, args, x.device,
+                        (x, residual, weight), ready)
 
 
 def astra_fused_add_rmsnorm(x: torch.Tensor, residual: torch.Tensor, weight: torch.Tensor,
@@ -239,8 +289,10 @@ def prepare_silu_and_mul(out: torch.Tensor, input: torch.Tensor) -> PreparedCall
         raise ValueError("input must be [T, 2*D]")
     T, D = input.shape[0], input.shape[1] // 2
     _check(out, "out", input.dtype, (T, D), input.device)
-    args = (_ptr(out), _ptr(input), ctypes.c_int64(T), ctypes.c_int64(D), ctypes.c_int(code))
-    return PreparedCall("astra_silu_and_mul", load_library().astra_silu_and_mul, args, input.device, (out, input))
+    args = lambda: (_ptr(out), _ptr(input), ctypes.c_int64(T), ctypes.c_int64(D), ctypes.c_int(code))  # noqa: E731
+    lib = load_library()
+    ready = _fast.prepare(_fast.KIND_SILU, (out.data_ptr(), input.data_ptr()), (T, D), 0.0, code, ())
+    return PreparedCall("astra_silu_and_mul", lib.astra_silu_and_mul, args, input.device, (out, input), ready)
 
 
 def astra_silu_and_mul(out: torch.Tensor, input: torch.Tensor,
@@ -264,10 +316,14 @@ def prepare_merge_attn_states_lse(v_out: torch.Tensor, lse_out: Optional[torch.T
     _check(lse_b, "lse_b", torch.float32, (T, Hh), v_a.device)
     if lse_out is not None:
         _check(lse_out, "lse_out", torch.float32, (T, Hh), v_a.device)
-    args = (_ptr(v_out), _ptr(lse_out), _ptr(v_a), _ptr(lse_a), _ptr(v_b), _ptr(lse_b),
-            ctypes.c_int64(T), ctypes.c_int64(Hh), ctypes.c_int64(D), ctypes.c_int(code))
-    return PreparedCall("astra_merge_attn_states_lse", load_library().astra_merge_attn_states_lse, args,
-                        v_a.device, (v_out, lse_out, v_a, lse_a, v_b, lse_b))
+    args = lambda: (_ptr(v_out), _ptr(lse_out), _ptr(v_a), _ptr(lse_a), _ptr(v_b), _ptr(lse_b),  # noqa: E731
+                    ctypes.c_int64(T), ctypes.c_int64(Hh), ctypes.c_int64(D), ctypes.c_int(code))
+    lib = load_library()
+    ready = _fast.prepare(_fast.KIND_MERGE,
+                          (v_out.data_ptr(), lse_out.data_ptr() if lse_out is not None else None, v_a.data_ptr(),
+                           lse_a.data_ptr(), v_b.data_ptr(), lse_b.data_ptr()), (T, Hh, D), 0.0, code, ())
+    return PreparedCall("astra_merge_attn_states_lse", lib.astra_merge_attn_states_lse, args,
+                        v_a.device, (v_out, lse_out, v_a, lse_a, v_b, lse_b), ready)
 
 
 def astra_merge_attn_states_lse(v_out: torch.Tensor, lse_out: Optional[torch.Tensor],
@@ -294,11 +350,14 @@ def prepare_fused_allreduce_add_rmsnorm(y: torch.Tensor, residual: torch.Tensor,
     for i, p in enumerate(parts):
         # a partial may sit on another GPU (that is the point of the call): no device check here
         _check(p, f"parts[{i}]", y.dtype, (T, H))
-    table = (ctypes.c_void_p * len(parts))(*[p.data_ptr() for p in parts])
-    args = (_ptr(y), _ptr(residual), table, ctypes.c_int(len(parts)), _ptr(weight), ctypes.c_int64(T),
-            ctypes.c_int64(H), ctypes.c_float(float(eps)), ctypes.c_int(code))
-    return PreparedCall("astra_fused_allreduce_add_rmsnorm", load_library().astra_fused_allreduce_add_rmsnorm,
-                        args, y.device, (y, residual, weight, table, *parts))
+    args = lambda: (_ptr(y), _ptr(residual), (ctypes.c_void_p * len(parts))(*[p.data_ptr() for p in parts]),  # noqa: E731
+                    ctypes.c_int(len(parts)), _ptr(weight), ctypes.c_int64(T), ctypes.c_int64(H),
+                    ctypes.c_float(float(eps)), ctypes.c_int(code))
+    lib = load_library()
+    ready = _fast.prepare(_fast.KIND_ALLREDUCE_RMSNORM, (y.data_ptr(), residual.data_ptr(), weight.data_ptr()),
+                          (T, H), float(eps), code, tuple(p.data_ptr() for p in parts))
+    return PreparedCall("astra_fused_allreduce_add_rmsnorm", lib.astra_fused_allreduce_add_rmsnorm,
+                        args, y.device, (y, residual, weight, *parts), ready)
 
 
 def astra_fused_allreduce_add_rmsnorm(y: torch.Tensor, residual: torch.Tensor, parts, weight: torch.Tensor,

@@ -1,6 +1,8 @@
-"""Build ``libastra.so`` (the CUDA kernels and their C ABI) for sm_100a with nvcc.
+"""Build ``libastra.so`` (the CUDA kernels and their C ABI) for sm_100a with nvcc, the ablation
+library beside it, and ``_astra_fastcall`` (a small CPython extension that re-issues prepared calls
+without ctypes) with the host C compiler.
 
-Usage: ``python -m paper_2509_07506_b200.build [--force]``.  The shared object is written next
+Usage: ``python -m paper_2509_07506_b200.build [--force]``.  The shared objects are written next
 to this file; nothing is installed outside the source tree.
 """
 from __future__ import annotations
@@ -11,6 +13,7 @@ import re
 import shutil
 import subprocess
 import sys
+import sysconfig
 
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
@@ -18,9 +21,11 @@ CSRC = os.path.join(PKG_DIR, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB_PATH = os.path.join(PKG_DIR, "libastra.so")
 ABLATION_LIB_PATH = os.path.join(PKG_DIR, "libastra_ablation.so")
+FASTCALL_PATH = os.path.join(PKG_DIR, "_astra_fastcall.so")
 
 SOURCES = ["astra.cu", "astra_allreduce.cu"]
 ABLATION_SOURCES = ["ablation.cu"]
+FASTCALL_SOURCES = ["fastcall.c"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
     "-O3", "-std=c++17", "-lineinfo",
@@ -39,7 +44,7 @@ def _nvcc() -> str:
 
 def _inputs():
     files = [os.path.join(INCLUDE, f) for f in os.listdir(INCLUDE) if f.endswith(".h")]
-    files += [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh", ".h"))]
+    files += [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh", ".h", ".c"))]
     return files
 
 
@@ -92,8 +97,27 @@ def _compile(lib_path: str, sources, force: bool, verbose: bool, extra_flags=())
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile libastra.so if it is missing or was built from other sources; returns its path."""
+    """Compile libastra.so (and the _astra_fastcall extension the binding loads with it) if missing or
+    built from other sources; returns the library's path."""
+    build_fastcall(force)
     return _compile(LIB_PATH, SOURCES, force, verbose)
+
+
+def build_fastcall(force: bool = False) -> str:
+    """Compile the _astra_fastcall extension (plain C against the CPython headers) if it is missing
+    or was built from other sources; returns its path."""
+    if not force and not is_stale(FASTCALL_PATH):
+        return FASTCALL_PATH
+    cc = shutil.which("gcc") or shutil.which("cc")
+    if cc is None:
+        raise RuntimeError("no C compiler found: _astra_fastcall cannot be built")
+    tmp = FASTCALL_PATH + f".tmp{os.getpid()}"
+    cmd = [cc, "-O2", "-std=c11", "-fPIC", "-shared", "-fvisibility=hidden", f'-DASTRA_BUILD_ID="{source_hash()}"',
+           "-I", sysconfig.get_paths()["include"], "-I", INCLUDE, "-o", tmp]
+    cmd += [os.path.join(CSRC, s) for s in FASTCALL_SOURCES]
+    subprocess.check_call(cmd)
+    os.replace(tmp, FASTCALL_PATH)
+    return FASTCALL_PATH
 
 
 def ensure_built(ablation: bool = False) -> str:
@@ -117,4 +141,5 @@ def build_ablation(force: bool = False, verbose: bool = False) -> str:
 
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(FASTCALL_PATH)
     print(build_ablation(force="--force" in sys.argv, verbose="-v" in sys.argv))

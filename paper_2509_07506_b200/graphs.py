@@ -1,7 +1,7 @@
 """Replaying a fixed sequence of calls from a CUDA graph.
 
 For decode-sized batches every call of this library is bound by launch cost, not by the GPU: a
-prepared call costs about 3.5 us of host time for 1-2 us of device time.  A sequence of prepared
+prepared call costs 2.5-3 us of host time for 1-2 us of device time.  A sequence of prepared
 calls on fixed tensors (a layer's add+norm, activation and merge, say) can be captured once into a
 CUDA graph and replayed with a single launch; the kernels keep their programmatic-dependent-launch
 edges inside the graph, so each one's prologue (and its L2 prefetch) overlaps the previous one's tail.

@@ -407,3 +407,69 @@ int main(void) {
                            str(src), "-o", str(exe), "-L", libdir, "-lastra", f"-Wl,-rpath,{libdir}"])
     out = subprocess.run([str(exe)], capture_output=True, text=True)
     assert out.returncode == 0 and out.stdout.strip() == "ok"
+
+
+# ---- the _astra_fastcall extension (prepared calls re-issued without ctypes) --------------------
+
+def test_fastcall_module_launches_what_ctypes_launches(lib):
+    """The extension hands a prepared struct to the same entry points: for fake addresses (nothing
+    can be launched on a machine without a GPU, and every argument error is reported first) each
+    status equals the one the ctypes call returns for the same arguments."""
+    fast = binding._fast
+    assert fast is not None and fast.build_id() == astra_build.source_hash()
+    cases = [
+        (fast.KIND_RMSNORM, lib.astra_fused_add_rmsnorm, (A, 2 * A, 3 * A), (4, 64), 1e-6, 0, ()),
+        (fast.KIND_RMSNORM, lib.astra_fused_add_rmsnorm, (A, A, 3 * A), (4, 64), 1e-6, 0, ()),          # overlap
+        (fast.KIND_RMSNORM, lib.astra_fused_add_rmsnorm, (A + 1, 2 * A, 3 * A), (4, 64), 1e-6, 1, ()),  # misaligned
+        (fast.KIND_RMSNORM, lib.astra_fused_add_rmsnorm, (A, 2 * A, 3 * A), (4, 0), 1e-6, 0, ()),       # bad shape
+        (fast.KIND_RMSNORM, lib.astra_fused_add_rmsnorm, (None, None, None), (0, 64), 1e-6, 2, ()),     # empty batch
+        (fast.KIND_SILU, lib.astra_silu_and_mul, (A, 2 * A), (4, 64), 0.0, 0, ()),
+        (fast.KIND_SILU, lib.astra_silu_and_mul, (A, 2 * A), (4, 64), 0.0, 7, ()),                      # bad dtype
+        (fast.KIND_SILU, lib.astra_silu_and_mul, (A, None), (4, 64), 0.0, 0, ()),                       # NULL
+        (fast.KIND_MERGE, lib.astra_merge_attn_states_lse, (A, 2 * A, 3 * A, 4 * A, 5 * A, 6 * A), (4, 8, 64), 0.0, 0, ()),
+        (fast.KIND_MERGE, lib.astra_merge_attn_states_lse, (A, None, 3 * A, 4 * A, 5 * A, 6 * A), (4, 8, 64), 0.0, 1, ()),
+        (fast.KIND_MERGE, lib.astra_merge_attn_states_lse, (A, 4 * A, 3 * A, 4 * A, 5 * A, 6 * A), (4, 8, 64), 0.0, 0, ()),
+    ]
+    seen = set()
+    for kind, fn, ptrs, ext, eps, dtype, parts in cases:
+        ready = fast.prepare(kind, ptrs, ext, eps, dtype, parts)
+        if kind == fast.KIND_RMSNORM:
+            want = fn(*ptrs, *ext, eps, dtype, None)
+        else:
+            want = fn(*ptrs, *ext, dtype, None)
+        got = fast.launch(ready, 0)
+        assert got == want, (kind, ptrs, ext, dtype, got, want)
+        seen.add(got)
+    assert {binding.ASTRA_OK, binding.ASTRA_ERR_NULL_POINTER, binding.ASTRA_ERR_BAD_SHAPE, binding.ASTRA_ERR_BAD_DTYPE,
+            binding.ASTRA_ERR_MISALIGNED, binding.ASTRA_ERR_OVERLAP} <= seen
+    # the all-reduce form: the table of partials lives in the prepared struct
+    table = (ctypes.c_void_p * 3)(4 * A, 5 * A, 6 * A)
+    want = lib.astra_fused_allreduce_add_rmsnorm(A, 2 * A, table, 3, 3 * A, 4, 64, 1e-6, 0, None)
+    got = fast.launch(fast.prepare(fast.KIND_ALLREDUCE_RMSNORM, (A, 2 * A, 3 * A), (4, 64), 1e-6, 0, (4 * A, 5 * A, 6 * A)), 0)
+    assert got == want
+    table = (ctypes.c_void_p * 2)(4 * A, A)   # a partial that is the output
+    want = lib.astra_fused_allreduce_add_rmsnorm(A, 2 * A, table, 2, 3 * A, 4, 64, 1e-6, 0, None)
+    got = fast.launch(fast.prepare(fast.KIND_ALLREDUCE_RMSNORM, (A, 2 * A, 3 * A), (4, 64), 1e-6, 0, (4 * A, A)), 0)
+    assert got == want == binding.ASTRA_ERR_OVERLAP
+
+
+def test_fastcall_module_refuses_malformed_preparations(lib):
+    fast = binding._fast
+    with pytest.raises(ValueError):
+        fast.prepare(9, (A,), (1,), 0.0, 0, ())
+    with pytest.raises(ValueError):
+        fast.prepare(fast.KIND_SILU, (A, 2 * A, 3 * A), (4, 64), 0.0, 0, ())       # three pointers for a two-pointer call
+    with pytest.raises(ValueError):
+        fast.prepare(fast.KIND_MERGE, (A,) * 6, (4, 64), 0.0, 0, ())              # two extents for a three-extent call
+    with pytest.raises(ValueError):
+        fast.prepare(fast.KIND_RMSNORM, (A, 2 * A, 3 * A), (4, 64), 0.0, 0, (A,))  # partials on a call without any
+    with pytest.raises(ValueError):
+        fast.prepare(fast.KIND_ALLREDUCE_RMSNORM, (A, 2 * A, 3 * A), (4, 64), 0.0, 0, ())
+    with pytest.raises(ValueError):
+        fast.prepare(fast.KIND_ALLREDUCE_RMSNORM, (A, 2 * A, 3 * A), (4, 64), 0.0, 0, (A,) * 17)
+    with pytest.raises(TypeError):
+        fast.prepare(fast.KIND_SILU, (A, "x"), (4, 64), 0.0, 0, ())
+    with pytest.raises(TypeError):
+        fast.launch(object(), 0)
+    with pytest.raises(TypeError):
+        fast.Prepared()

@@ -386,6 +386,44 @@ def test_prepared_calls_match_plain_calls_bit_for_bit():
     check_values(f64(x2.cpu()), oy, BF16, what="prepared rmsnorm")
 
 
+def test_prepared_call_routes_agree_bit_for_bit():
+    """A prepared call is issued by the extension module; ``via_ctypes`` issues the same arguments
+    through ctypes.  Both reach the same entry point: identical bits, on the current and a side stream."""
+    rms = wl.rmsnorm_inputs(40, 5120, FP16, eps=1e-5, seed=41)
+    mi = wl.merge_inputs(70, 8, 128, BF16, seed=43, neg_inf_frac=0.05)
+    ar = wl.allreduce_rmsnorm_inputs(24, 4096, 3, BF16, seed=44)
+    w = rms.weight.cuda()
+    va, vb, sa, sb = mi.v_a.cuda(), mi.v_b.cuda(), mi.lse_a.cuda(), mi.lse_b.cuda()
+    parts, aw = [p.cuda() for p in ar.parts], ar.weight.cuda()
+    outs = []
+    side = torch.cuda.Stream()
+    for route in ("extension", "ctypes", "ctypes on a side stream"):
+        x, r = rms.x.cuda(), rms.residual.cuda()
+        vo, lo = torch.empty_like(va), torch.empty_like(sa)
+        y, rr = torch.empty_like(parts[0]), ar.residual.cuda()
+        calls = [astra.prepare_fused_add_rmsnorm(x, r, w, rms.eps), astra.prepare_merge_attn_states_lse(vo, lo, va, sa, vb, sb),
+                 astra.prepare_fused_allreduce_add_rmsnorm(y, rr, parts, aw, ar.eps)]
+        if route == "extension":
+            for c in calls:
+                c()
+        elif route == "ctypes":
+            for c in calls:
+                c.via_ctypes()
+        else:
+            side.wait_stream(torch.cuda.current_stream())
+            for c in calls:
+                c.via_ctypes(side)
+            torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        outs.append((x, r, vo, lo.view(torch.int32), y, rr))
+    for other in outs[1:]:
+        for a, b in zip(outs[0], other):
+            assert torch.equal(a, b)
+    oy, orr = oracle.fused_add_rmsnorm(wl.bits(rms.x), wl.bits(rms.residual), wl.bits(rms.weight), rms.eps, FP16)
+    assert np.array_equal(wl.bits(outs[0][1].cpu()), orr)
+    check_values(f64(outs[0][0].cpu()), oy, FP16, what="prepared rmsnorm, extension route")
+
+
 def test_decode_chain_replayed_from_a_graph_matches_the_oracle():
     """The three calls at a decode-sized batch, captured once and replayed with new inputs: every
     replay's outputs are compared with the oracle (and are bit-identical to the eager calls')."""
