@@ -602,6 +602,24 @@ def allreduce_variants(astra, dev, peak) -> list:
                 row.update(fractions(gbs, peak))
             rows.append(row)
             del sets
+    # Two-shot form: one rank's call on its block of T / N rows, the results stored to N destinations
+    # each (all of them in this GPU's memory here; over NVLink N - 1 of the N would be peer stores).
+    T = wl.CHAIN_T
+    for n in (2, 4, 8):
+        Tb = T // n
+        nbytes = wl.two_shot_rmsnorm_bytes(Tb, H, n, n, n)
+        make = lambda: ([torch.randn((Tb, H), device=dev).to(td) for _ in range(n)], torch.randn((Tb, H), device=dev).to(td),  # noqa: E731
+                        [torch.empty((Tb, H), device=dev, dtype=td) for _ in range(n)],
+                        [torch.empty((Tb, H), device=dev, dtype=td) for _ in range(n - 1)], torch.ones((H,), device=dev, dtype=td))
+        sets = _rotating(make, nbytes)
+        call = lambda b: astra.astra_fused_allreduce_add_rmsnorm_ex(b[2], [b[1]] + b[3], b[1], b[0], b[4], 1e-5)  # noqa: E731
+        us = _time_graph(call, sets)
+        gbs = nbytes / us / 1e3
+        rows.append({"form": "two-shot: one rank's row block, results stored to every rank's buffers",
+                     "shape": [Tb, H], "of_batch": [T, H], "n_parts": n, "n_destinations": n,
+                     "algorithmic_bytes": nbytes, "us_device": round(us, 2), "gbs": round(gbs, 1),
+                     **(fractions(gbs, peak) if nbytes > 2 * L2_BYTES else {})})
+        del sets
     return rows
 
 

@@ -187,6 +187,36 @@ astra_status_t astra_fused_allreduce_add_rmsnorm(void *y, void *residual,
                                                  const void *weight, int64_t T, int64_t H, float eps,
                                                  astra_dtype_t dtype, void *cuda_stream);
 
+/*
+ * fused_allreduce_add_rmsnorm with several destinations per result: the two-shot form of the same
+ * operation (Table 1, Kernel 2 on a hidden state given as n_parts partial sums; arithmetic exactly
+ * as astra_fused_allreduce_add_rmsnorm).  For batches large enough that reading every partial on
+ * every rank would be bound by the links, each rank calls this for ITS OWN BLOCK OF ROWS only and
+ * has the results stored into every rank's buffers, so that each element crosses the links once as
+ * a partial and once as a result:
+ *
+ *   y_outs         HOST array of n_y device pointers; each receives the T normalised rows.
+ *   residual_outs  HOST array of n_r device pointers; each receives the T rows of the new residual.
+ *   residual       [T, H] in: r.  One of residual_outs may be exactly this pointer (in place).
+ *   x_parts, n_parts, weight, T, H, eps, dtype: as in astra_fused_allreduce_add_rmsnorm.
+ *   n_y, n_r       1 .. 16 each (else ASTRA_ERR_BAD_SHAPE).
+ *
+ * All tensors are dense [T, H] blocks; the caller passes pointers already advanced to the block's
+ * first row in each buffer.  A destination may live in another GPU's memory mapped into this
+ * process: it is written with ordinary per-thread stores only.  With n_y = n_r = 1 and
+ * residual_outs[0] = residual this is astra_fused_allreduce_add_rmsnorm, bit for bit.
+ * Ordering is the caller's, in both directions: the call waits for nothing, and the ranks that own
+ * the destinations must not read them before this kernel has completed.
+ * Every destination must not overlap any other destination, any partial, weight, or residual
+ * (except the exact in-place case above): ASTRA_ERR_OVERLAP.
+ */
+astra_status_t astra_fused_allreduce_add_rmsnorm_ex(void *const *y_outs, int32_t n_y,
+                                                    void *const *residual_outs, int32_t n_r,
+                                                    const void *residual,
+                                                    const void *const *x_parts, int32_t n_parts,
+                                                    const void *weight, int64_t T, int64_t H, float eps,
+                                                    astra_dtype_t dtype, void *cuda_stream);
+
 /* Static, NUL-terminated description of a status code (never NULL). */
 const char *astra_status_string(astra_status_t status);
 

@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     PreparedCall,
     astra_fused_add_rmsnorm,
     astra_fused_allreduce_add_rmsnorm,
+    astra_fused_allreduce_add_rmsnorm_ex,
     prepare_fused_add_rmsnorm,
     prepare_fused_allreduce_add_rmsnorm,
     prepare_merge_attn_states_lse,

@@ -37,6 +37,7 @@ EXPORTED_SYMBOLS = (
     "astra_silu_and_mul_ex",
     "astra_merge_attn_states_lse_ex",
     "astra_fused_allreduce_add_rmsnorm",
+    "astra_fused_allreduce_add_rmsnorm_ex",
     "astra_status_string",
     "astra_build_id",
 )
@@ -79,6 +80,9 @@ def load_library() -> ctypes.CDLL:
     lib.astra_merge_attn_states_lse_ex.restype = i32
     lib.astra_fused_allreduce_add_rmsnorm.argtypes = [vp, vp, ctypes.POINTER(vp), i32, vp, i64, i64, f32, i32, vp]
     lib.astra_fused_allreduce_add_rmsnorm.restype = i32
+    lib.astra_fused_allreduce_add_rmsnorm_ex.argtypes = [ctypes.POINTER(vp), i32, ctypes.POINTER(vp), i32, vp,
+                                                         ctypes.POINTER(vp), i32, vp, i64, i64, f32, i32, vp]
+    lib.astra_fused_allreduce_add_rmsnorm_ex.restype = i32
     lib.astra_status_string.argtypes = [i32]
     lib.astra_status_string.restype = ctypes.c_char_p
     lib.astra_build_id.argtypes = []
@@ -368,6 +372,37 @@ def astra_fused_allreduce_add_rmsnorm(y: torch.Tensor, residual: torch.Tensor, p
     memory this process can address; y, residual and weight live on the GPU that runs the kernel.
     The call waits for nothing: order it after the partials have been written."""
     prepare_fused_allreduce_add_rmsnorm(y, residual, parts, weight, eps)(stream)
+
+
+def astra_fused_allreduce_add_rmsnorm_ex(y_outs, residual_outs, residual: torch.Tensor, parts, weight: torch.Tensor,
+                                         eps: float, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Two-shot form: this rank's block of rows [T, H] is reduced over ``parts`` (rank order, binary32,
+    the residual last) and normalised once, and the results are stored to every tensor of ``y_outs``
+    (the normalised rows) and of ``residual_outs`` (the new residual; one of them may be ``residual``
+    itself).  All tensors are the [T, H] row block, i.e. slices ``buf[first:first + T]`` of the ranks'
+    full buffers.  ``residual`` and ``weight`` live on the GPU that runs the kernel; partials and
+    destinations may live on other GPUs whose memory this process can address.  The call waits for
+    nothing and the destinations' owners must not read them before it has completed."""
+    parts, y_outs, residual_outs = list(parts), list(y_outs), list(residual_outs)
+    _check(residual, "residual")
+    code = _code(residual, "residual")
+    if residual.dim() != 2:
+        raise ValueError("residual must be [T, H]")
+    T, H = residual.shape
+    _check(weight, "weight", residual.dtype, (H,), residual.device)
+    for what, seq in (("parts", parts), ("y_outs", y_outs), ("residual_outs", residual_outs)):
+        if not 1 <= len(seq) <= 16:
+            raise ValueError(f"between 1 and 16 tensors are supported in {what}, got {len(seq)}")
+        for i, t in enumerate(seq):
+            # partials and destinations may sit on other GPUs (that is the point of the call): no device check
+            _check(t, f"{what}[{i}]", residual.dtype, (T, H))
+    table = lambda seq: (ctypes.c_void_p * len(seq))(*[t.data_ptr() for t in seq])  # noqa: E731
+    with _on_device(residual):
+        st = load_library().astra_fused_allreduce_add_rmsnorm_ex(
+            table(y_outs), len(y_outs), table(residual_outs), len(residual_outs), residual.data_ptr(),
+            table(parts), len(parts), weight.data_ptr(), T, H, float(eps), code, _stream(residual, stream))
+    if st != ASTRA_OK:
+        raise AstraError(st, "astra_fused_allreduce_add_rmsnorm_ex")
 
 
 # ---- strided / out-of-place forms ---------------------------------------------------------------

@@ -82,10 +82,12 @@ cudaError_t launch_rows(AllreduceOperands op, const uint16_t *w, int64_t T, int 
     for (int64_t t0 = 0; t0 < T; t0 += rows_per_launch) {
         const unsigned rows = static_cast<unsigned>(T - t0 < rows_per_launch ? T - t0 : rows_per_launch);
         AllreduceOperands o = op;
-        for (int p = 0; p < op.n_parts; ++p) o.part[p] += t0 * row_units;
+        for (int p = 0; p < kMaxParts; ++p) {  // unused slots repeat slot 0, so every slot moves along
+            o.part[p] += t0 * row_units;
+            o.y_out[p] += t0 * row_units;
+            o.r_out[p] += t0 * row_units;
+        }
         o.r += t0 * row_units;
-        o.y += t0 * row_units;
-        o.r_out += t0 * row_units;
         cudaError_t err;
         switch (vpt) {
             case 0: err = launch(fused_allreduce_add_rmsnorm_twopass_kernel<DT, VEC, GROUP>, rows, sweep_threads,
@@ -122,14 +124,79 @@ template <int DT>
 cudaError_t dispatch(const AllreduceOperands &op, const uint16_t *w, int64_t T, int H, float eps,
                      cudaStream_t stream) {
     VecPick pick(8);
-    pick.extent(static_cast<int64_t>(H) * Storage<DT>::UNITS).pointer(op.r).pointer(op.y).pointer(op.r_out).pointer(w);
+    pick.extent(static_cast<int64_t>(H) * Storage<DT>::UNITS).pointer(op.r).pointer(w);
     for (int p = 0; p < op.n_parts; ++p) pick.pointer(op.part[p]);
+    for (int d = 0; d < op.n_y; ++d) pick.pointer(op.y_out[d]);
+    for (int d = 0; d < op.n_r; ++d) pick.pointer(op.r_out[d]);
     switch (pick.vec) {
         case 8: return choose_shape<DT, 8>(op, w, T, H, eps, stream);
         case 4: return choose_shape<DT, 4>(op, w, T, H, eps, stream);
         case 2: return choose_shape<DT, 2>(op, w, T, H, eps, stream);
         default: return choose_shape<DT, 1>(op, w, T, H, eps, stream);
     }
+}
+
+// Shared by the two entry points.  y_outs / r_outs: n_y / n_r destinations of the normalised rows and
+// of the new residual; `residual` is the residual input, which one of r_outs may be exactly.
+astra_status_t allreduce_entry(void *const *y_outs, int32_t n_y, void *const *r_outs, int32_t n_r,
+                               const void *residual, const void *const *x_parts, int32_t n_parts,
+                               const void *weight, int64_t T, int64_t H, float eps, astra_dtype_t dtype,
+                               void *cuda_stream) {
+    if (!valid_dtype(dtype)) return ASTRA_ERR_BAD_DTYPE;
+    const int64_t U = units_per_elem(dtype);
+    if (n_parts < 1 || n_parts > kMaxParts || n_y < 1 || n_y > kMaxParts || n_r < 1 || n_r > kMaxParts)
+        return ASTRA_ERR_BAD_SHAPE;
+    if (T < 0 || H <= 0 || H > kMaxRowUnits / U) return ASTRA_ERR_BAD_SHAPE;
+    if (T > 0 && H > kInt64Max / 4 / T) return ASTRA_ERR_BAD_SHAPE;
+    if (T == 0) return ASTRA_OK;
+    if (!y_outs || !r_outs || !residual || !x_parts || !weight) return ASTRA_ERR_NULL_POINTER;
+    for (int p = 0; p < n_parts; ++p)
+        if (!x_parts[p]) return ASTRA_ERR_NULL_POINTER;
+    for (int d = 0; d < n_y; ++d)
+        if (!y_outs[d]) return ASTRA_ERR_NULL_POINTER;
+    for (int d = 0; d < n_r; ++d)
+        if (!r_outs[d]) return ASTRA_ERR_NULL_POINTER;
+    const size_t eb = static_cast<size_t>(2 * U);
+    if (!aligned(residual, eb) || !aligned(weight, eb)) return ASTRA_ERR_MISALIGNED;
+    for (int p = 0; p < n_parts; ++p)
+        if (!aligned(x_parts[p], eb)) return ASTRA_ERR_MISALIGNED;
+    for (int d = 0; d < n_y; ++d)
+        if (!aligned(y_outs[d], eb)) return ASTRA_ERR_MISALIGNED;
+    for (int d = 0; d < n_r; ++d)
+        if (!aligned(r_outs[d], eb)) return ASTRA_ERR_MISALIGNED;
+    // Every destination overlaps nothing else, except that a residual destination may be exactly the
+    // residual input.  (Memory of another GPU has addresses in the same unified space, so the
+    // byte-range test is meaningful for it too.)  Partials may overlap one another: they are only read.
+    const int64_t bytes = T * H * U * 2, wbytes = H * U * 2;
+    void *outs[2 * kMaxParts];
+    int n_out = 0;
+    for (int d = 0; d < n_y; ++d) outs[n_out++] = y_outs[d];
+    for (int d = 0; d < n_r; ++d) outs[n_out++] = r_outs[d];
+    for (int a = 0; a < n_out; ++a) {
+        const bool is_residual_dest = a >= n_y;
+        if (overlaps(outs[a], bytes, weight, wbytes)) return ASTRA_ERR_OVERLAP;
+        if (!(is_residual_dest && outs[a] == residual) && overlaps(outs[a], bytes, residual, bytes))
+            return ASTRA_ERR_OVERLAP;
+        for (int p = 0; p < n_parts; ++p)
+            if (overlaps(outs[a], bytes, x_parts[p], bytes)) return ASTRA_ERR_OVERLAP;
+        for (int b = a + 1; b < n_out; ++b)
+            if (overlaps(outs[a], bytes, outs[b], bytes)) return ASTRA_ERR_OVERLAP;
+    }
+    AllreduceOperands op;
+    for (int p = 0; p < kMaxParts; ++p) {
+        op.part[p] = static_cast<const uint16_t *>(x_parts[p < n_parts ? p : 0]);
+        op.y_out[p] = static_cast<uint16_t *>(y_outs[p < n_y ? p : 0]);
+        op.r_out[p] = static_cast<uint16_t *>(r_outs[p < n_r ? p : 0]);
+    }
+    op.n_parts = n_parts;
+    op.n_y = n_y;
+    op.n_r = n_r;
+    op.r = static_cast<const uint16_t *>(residual);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const uint16_t *wp = static_cast<const uint16_t *>(weight);
+    cudaError_t err = cudaSuccess;
+    ASTRA_FOR_DTYPE(dtype, err = dispatch<DT>(op, wp, T, static_cast<int>(H), eps, stream));
+    return launch_status(err);
 }
 
 }  // namespace
@@ -139,41 +206,17 @@ extern "C" {
 astra_status_t astra_fused_allreduce_add_rmsnorm(void *y, void *residual, const void *const *x_parts,
                                                  int32_t n_parts, const void *weight, int64_t T, int64_t H,
                                                  float eps, astra_dtype_t dtype, void *cuda_stream) {
-    if (!valid_dtype(dtype)) return ASTRA_ERR_BAD_DTYPE;
-    const int64_t U = units_per_elem(dtype);
-    if (n_parts < 1 || n_parts > kMaxParts) return ASTRA_ERR_BAD_SHAPE;
-    if (T < 0 || H <= 0 || H > kMaxRowUnits / U) return ASTRA_ERR_BAD_SHAPE;
-    if (T > 0 && H > kInt64Max / 4 / T) return ASTRA_ERR_BAD_SHAPE;
-    if (T == 0) return ASTRA_OK;
-    if (!y || !residual || !x_parts || !weight) return ASTRA_ERR_NULL_POINTER;
-    for (int p = 0; p < n_parts; ++p)
-        if (!x_parts[p]) return ASTRA_ERR_NULL_POINTER;
-    const size_t eb = static_cast<size_t>(2 * U);
-    if (!aligned(y, eb) || !aligned(residual, eb) || !aligned(weight, eb)) return ASTRA_ERR_MISALIGNED;
-    for (int p = 0; p < n_parts; ++p)
-        if (!aligned(x_parts[p], eb)) return ASTRA_ERR_MISALIGNED;
-    // The two outputs overlap nothing else.  (A partial in another GPU's memory has an address in
-    // the same unified space, so the byte-range test is meaningful for it too.)  Partials may
-    // overlap one another: they are only read.
-    const int64_t bytes = T * H * U * 2, wbytes = H * U * 2;
-    if (overlaps(y, bytes, residual, bytes) || overlaps(y, bytes, weight, wbytes) ||
-        overlaps(residual, bytes, weight, wbytes))
-        return ASTRA_ERR_OVERLAP;
-    for (int p = 0; p < n_parts; ++p)
-        if (overlaps(y, bytes, x_parts[p], bytes) || overlaps(residual, bytes, x_parts[p], bytes))
-            return ASTRA_ERR_OVERLAP;
-    AllreduceOperands op;
-    for (int p = 0; p < kMaxParts; ++p)
-        op.part[p] = static_cast<const uint16_t *>(x_parts[p < n_parts ? p : 0]);
-    op.n_parts = n_parts;
-    op.r = static_cast<const uint16_t *>(residual);
-    op.r_out = static_cast<uint16_t *>(residual);
-    op.y = static_cast<uint16_t *>(y);
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const uint16_t *wp = static_cast<const uint16_t *>(weight);
-    cudaError_t err = cudaSuccess;
-    ASTRA_FOR_DTYPE(dtype, err = dispatch<DT>(op, wp, T, static_cast<int>(H), eps, stream));
-    return launch_status(err);
+    void *ys[1] = {y}, *rs[1] = {residual};  // one destination apiece, the residual in place
+    return allreduce_entry(ys, 1, rs, 1, residual, x_parts, n_parts, weight, T, H, eps, dtype, cuda_stream);
+}
+
+astra_status_t astra_fused_allreduce_add_rmsnorm_ex(void *const *y_outs, int32_t n_y, void *const *residual_outs,
+                                                    int32_t n_r, const void *residual,
+                                                    const void *const *x_parts, int32_t n_parts,
+                                                    const void *weight, int64_t T, int64_t H, float eps,
+                                                    astra_dtype_t dtype, void *cuda_stream) {
+    return allreduce_entry(y_outs, n_y, residual_outs, n_r, residual, x_parts, n_parts, weight, T, H, eps, dtype,
+                           cuda_stream);
 }
 
 }  // extern "C"

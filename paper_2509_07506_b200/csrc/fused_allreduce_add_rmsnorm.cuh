@@ -4,14 +4,18 @@
 // Every addition is one binary32 addition, in rank order, the residual last, so that all ranks of a
 // group that run this on the same partials produce identical bits.
 //
-// This is the "one-shot" all-reduce: each rank reads all N partials of the rows it normalises (its
-// own from local memory, the others through peer-mapped addresses) and never writes to a peer.
-// All loads are plain per-thread `ld.global` (no multicast, no bulk or tensor-map copies), so a
-// partial may live in another GPU's memory.  The kernel waits for nothing: the caller orders it
-// after every rank has finished writing its partial (stream events, a host barrier).
+// One-shot form: each rank reads all N partials of the rows it normalises (its own from local
+// memory, the others through peer-mapped addresses) and writes only its own memory.  Two-shot form
+// (for batches large enough that the N-fold read would be bound by the links): each rank does this
+// for its own block of rows only and stores the results to every rank's buffers, so each element
+// crosses the links once as a partial and once as a result instead of N - 1 times.
+// All loads and stores are plain per-thread `ld.global` / `st.global` (no multicast, no bulk or
+// tensor-map copies), so a partial or a destination may live in another GPU's memory.  The kernel
+// waits for nothing: the caller orders it after every rank has finished writing its partial and
+// orders the consumers after it (stream events, a host barrier).
 //
-// HBM/NVLink-bound: (N + 3) * 2 bytes per element of 16-bit storage (N partials and r read, y and
-// r_out written).  One block owns a row and keeps the running binary32 sums in registers; the
+// HBM/NVLink-bound: (N + 1 + Dy + Dr) * 2 bytes per element of 16-bit storage (N partials and r read,
+// y written to Dy destinations and the new residual to Dr; N + 3 in the one-shot form).  One block owns a row and keeps the running binary32 sums in registers; the
 // partials are fetched GROUP at a time so that GROUP (+1 for the residual) vector loads per vector
 // position are in flight before the first addition (GROUP = 2 measured best; see the launch code).
 #pragma once
@@ -22,15 +26,30 @@ namespace astra {
 
 constexpr int kMaxParts = 16;
 
-// Dense [T, H] operands (row pitch = H).  Pointers are in 16-bit units.  r_out may be exactly r
-// (each thread reads the residual vectors it later overwrites); y overlaps nothing.
+// Dense [T, H] operands (row pitch = H).  Pointers are in 16-bit units.  Each result goes to one or
+// more destinations (the same bytes to each): with one destination apiece this is the one-shot
+// all-reduce; with one destination per rank it is the two-shot form, in which a rank reduces and
+// normalises only its own row block and pushes the results into every rank's buffers.  A residual
+// destination may be exactly r (each thread reads the residual vectors it later overwrites); the
+// destinations overlap nothing else.
 struct AllreduceOperands {
     const uint16_t *part[kMaxParts];  // rank order
     const uint16_t *r;
-    uint16_t *y;
-    uint16_t *r_out;
-    int n_parts;
+    uint16_t *y_out[kMaxParts];
+    uint16_t *r_out[kMaxParts];
+    int n_parts, n_y, n_r;
 };
+
+// The same vector to each of the first n destinations, with plain per-thread stores (a destination
+// may be another GPU's memory).  Unrolled and left by a break, so every copy has a constant index.
+template <int UV>
+__device__ __forceinline__ void store_to_all(uint16_t *const (&dst)[kMaxParts], int n, int64_t at, const Pack<UV> &v) {
+#pragma unroll
+    for (int d = 0; d < kMaxParts; ++d) {
+        if (d >= n) break;
+        store<UV, St::Stream>(dst[d] + at, v);
+    }
+}
 
 // s += x, two elements per instruction where the vector length is even (same roundings as scalar adds).
 template <int VEC>
@@ -142,7 +161,7 @@ fused_allreduce_add_rmsnorm_reg_kernel(const __grid_constant__ AllreduceOperands
             float fr[VEC];
             widen<DT, VEC>(pr[i], fr);
             add_and_square(s[i], fr, s[i], acc, acc2);  // the residual joins last
-            store<UV, St::Stream>(op.r_out + row + v * UV, narrow<DT, VEC>(s[i]));
+            store_to_all<UV>(op.r_out, op.n_r, row + v * UV, narrow<DT, VEC>(s[i]));
         }
     }
 
@@ -162,7 +181,7 @@ fused_allreduce_add_rmsnorm_reg_kernel(const __grid_constant__ AllreduceOperands
             float fw[VEC], fy[VEC];
             widen<DT, VEC>(pw[i], fw);
             scale(s[i], rstd, fw, fy);
-            store<UV, St::Stream>(op.y + row + v * UV, narrow<DT, VEC>(fy));
+            store_to_all<UV>(op.y_out, op.n_y, row + v * UV, narrow<DT, VEC>(fy));
         }
     }
 }
@@ -230,8 +249,8 @@ fused_allreduce_add_rmsnorm_twopass_kernel(const __grid_constant__ AllreduceOper
         widen<DT, VEC>(load<UV, Ld::Keep>(weight + static_cast<int64_t>(v) * UV), fw);
 #pragma unroll
         for (int k = 0; k < VEC; ++k) fy[k] = s[k] * rstd * fw[k];
-        store<UV, St::Stream>(op.r_out + at, narrow<DT, VEC>(s));
-        store<UV, St::Stream>(op.y + at, narrow<DT, VEC>(fy));
+        store_to_all<UV>(op.r_out, op.n_r, at, narrow<DT, VEC>(s));
+        store_to_all<UV>(op.y_out, op.n_y, at, narrow<DT, VEC>(fy));
     }
 }
 

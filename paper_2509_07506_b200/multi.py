@@ -123,10 +123,19 @@ def exchange_partials(local, export, open_remote, group=None) -> list:
     return [local if owner == rank else open_remote(handles[owner], owner) for owner in range(world)]
 
 
+def exchange_buffers(local, export, open_remote, group=None) -> list:
+    """The same exchange for any per-rank buffer: the two-shot form of the fused all-reduce
+    (astra_fused_allreduce_add_rmsnorm_ex) needs every rank's output buffers as well, because each rank
+    stores its block of normalised rows (and of the new residual) into all of them."""
+    return exchange_partials(local, export, open_remote, group)
+
+
 def row_block_of_rank(total_rows: int, group=None) -> Tuple[int, int]:
-    """After the fused all-reduce every rank needs the normalised rows it goes on to use.  With
-    sequence-parallel consumers each rank normalises only its own contiguous row block of the
-    [total_rows, H] hidden state (reading that block from all N partials): (first_row, row_count)."""
+    """The contiguous row block of the [total_rows, H] hidden state that this rank reduces and
+    normalises (reading that block from all N partials): (first_row, row_count).  Used two ways: with
+    sequence-parallel consumers the rank keeps the block for itself; in the two-shot form it stores
+    the block into every rank's buffers, so that all ranks end up with all rows while each element
+    crosses the links once as a partial and once as a result."""
     if not (dist.is_available() and dist.is_initialized()):
         return 0, total_rows
     return shard_rows(total_rows, dist.get_world_size(group), dist.get_rank(group))

@@ -233,6 +233,12 @@ def allreduce_rmsnorm_bytes(T: int, H: int, n_parts: int, elem: int = 2) -> int:
     return (n_parts + 3) * T * H * elem + H * elem
 
 
+def two_shot_rmsnorm_bytes(T_block: int, H: int, n_parts: int, n_y: int, n_r: int, elem: int = 2) -> int:
+    """The two-shot form on a block of rows: read the n_parts partials and r, write y to n_y
+    destinations and r' to n_r, read the weight once."""
+    return (n_parts + 1 + n_y + n_r) * T_block * H * elem + H * elem
+
+
 def silu_bytes(T: int, D: int, elem: int = 2) -> int:
     """Read gate and up, write out."""
     return 3 * T * D * elem

@@ -165,6 +165,48 @@ def test_allreduce_rmsnorm_argument_errors(lib):
         assert call(parts=(16 * A,), T=1, H=40000, y=32 * A, r=48 * A, w=64 * A) == binding.ASTRA_ERR_CUDA
 
 
+def test_allreduce_rmsnorm_ex_argument_errors(lib):
+    """The two-shot form: several destinations per result.  Every destination is checked for NULL,
+    alignment and overlap with every other operand; one residual destination may be the residual."""
+    import ctypes as C
+    f = lib.astra_fused_allreduce_add_rmsnorm_ex
+    R, W = 2 * A, 3 * A
+
+    def tab(ptrs):
+        return (C.c_void_p * max(1, len(ptrs)))(*ptrs) if ptrs is not None else None
+
+    def call(ys=(8 * A, 9 * A), rs=(R, 10 * A), r=R, parts=(4 * A, 5 * A), w=W, T=1, H=8, dtype=0, n_y=None, n_r=None):
+        return f(tab(ys), len(ys) if n_y is None else n_y, tab(rs), len(rs) if n_r is None else n_r, r,
+                 tab(parts), len(parts), w, T, H, 1e-6, dtype, None)
+
+    assert call(ys=None, n_y=1) == binding.ASTRA_ERR_NULL_POINTER
+    assert call(rs=None, n_r=1) == binding.ASTRA_ERR_NULL_POINTER
+    assert call(r=None) == binding.ASTRA_ERR_NULL_POINTER
+    assert call(ys=(8 * A, None)) == binding.ASTRA_ERR_NULL_POINTER
+    assert call(rs=(R, None)) == binding.ASTRA_ERR_NULL_POINTER
+    assert call(n_y=0) == binding.ASTRA_ERR_BAD_SHAPE
+    assert call(n_r=0) == binding.ASTRA_ERR_BAD_SHAPE
+    assert call(ys=tuple((20 + i) * A for i in range(17))) == binding.ASTRA_ERR_BAD_SHAPE
+    assert call(rs=tuple((20 + i) * A for i in range(17))) == binding.ASTRA_ERR_BAD_SHAPE
+    assert call(dtype=5) == binding.ASTRA_ERR_BAD_DTYPE
+    assert call(ys=(8 * A, 9 * A + 1)) == binding.ASTRA_ERR_MISALIGNED
+    assert call(rs=(R, 10 * A + 2), dtype=binding.ASTRA_FP32) == binding.ASTRA_ERR_MISALIGNED
+    assert call(ys=(8 * A, 8 * A)) == binding.ASTRA_ERR_OVERLAP          # two destinations, one address
+    assert call(ys=(8 * A, 10 * A)) == binding.ASTRA_ERR_OVERLAP         # a y destination over a residual destination
+    assert call(ys=(8 * A, R)) == binding.ASTRA_ERR_OVERLAP              # y over the residual input
+    assert call(rs=(R + 8, 10 * A)) == binding.ASTRA_ERR_OVERLAP         # a residual destination shifted into the residual
+    assert call(rs=(R, 5 * A)) == binding.ASTRA_ERR_OVERLAP              # a residual destination over a partial
+    assert call(ys=(8 * A, W + 4)) == binding.ASTRA_ERR_OVERLAP          # over the weight
+    assert call(T=0) == binding.ASTRA_OK
+    assert call(T=0, ys=None, rs=None, r=None, n_y=2, n_r=2) == binding.ASTRA_OK
+    import torch
+    if not torch.cuda.is_available():
+        assert call() == binding.ASTRA_ERR_CUDA                          # in place plus one more destination
+        assert call(rs=(10 * A, 11 * A)) == binding.ASTRA_ERR_CUDA        # no destination is the residual itself
+        assert call(ys=tuple((20 + i) * A for i in range(16)), rs=tuple((40 + i) * A for i in range(16)), T=3, H=4100) \
+            == binding.ASTRA_ERR_CUDA
+
+
 def test_silu_argument_errors(lib):
     f = lib.astra_silu_and_mul
     assert f(None, A, 1, 8, 0, None) == binding.ASTRA_ERR_NULL_POINTER

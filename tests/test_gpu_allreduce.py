@@ -118,6 +118,115 @@ def test_allreduce_rmsnorm_prepared_and_repeatable():
         assert torch.equal(ref[0], got[0]) and torch.equal(ref[1], got[1])
 
 
+# ---- the two-shot form: a rank reduces its own row block and stores the results to every rank ----
+
+def run_two_shot(inp: wl.AllreduceRmsnormInputs, world: int, rank: int, offset=0, in_place=True):
+    """One rank's call of the two-shot form on one GPU: `world` full-size [T, H] destination buffers
+    for y and for the residual stand for the ranks' buffers; the rank's own residual buffer (slot
+    `rank`) is the residual input when in_place.  Inside the rank's row block every destination must
+    hold the oracle's rows; outside it nothing may change."""
+    from paper_2509_07506_b200 import multi
+    T, H = inp.residual.shape
+    first, count = multi.shard_rows(T, world, rank)
+    sl = slice(first, first + count)
+    td = inp.residual.dtype
+    sentinel = torch.full((T, H), 7.0, dtype=td)
+    gparts = [Guarded(p, offset) for p in inp.parts]
+    gw = Guarded(inp.weight, offset)
+    gys = [Guarded(sentinel, offset) for _ in range(world)]
+    grs = [Guarded(inp.residual if (in_place and d == rank) else sentinel, offset) for d in range(world)]
+    gin = grs[rank] if in_place else Guarded(inp.residual, offset)
+    astra.astra_fused_allreduce_add_rmsnorm_ex([g.t[sl] for g in gys], [g.t[sl] for g in grs], gin.t[sl],
+                                               [g.t[sl] for g in gparts], gw.t, inp.eps)
+    torch.cuda.synchronize()
+    for g in gparts + gys + grs + [gw, gin]:
+        g.check()
+    for g, p in zip(gparts, inp.parts):
+        assert torch.equal(g.host().view(torch.uint8), p.view(torch.uint8)), "a partial was modified"
+    if count == 0:
+        oy = orr = None
+    else:
+        oy, orr = oracle.fused_allreduce_add_rmsnorm([wl.bits(p[sl]) for p in inp.parts], wl.bits(inp.residual[sl]),
+                                                     wl.bits(inp.weight), inp.eps, inp.dtype, nthreads=NCPU)
+    outside = torch.ones(T, dtype=torch.bool)
+    outside[sl] = False
+    stats = {}
+    y0 = gys[0].host()
+    for d in range(world):
+        y, r = gys[d].host(), grs[d].host()
+        assert torch.equal(y.view(torch.uint8), y0.view(torch.uint8)), "the y destinations differ"
+        assert bool((y[outside] == 7.0).all()), "y was written outside the rank's row block"
+        keep = inp.residual if (in_place and d == rank) else sentinel
+        assert torch.equal(r[outside].view(torch.uint8), keep[outside].view(torch.uint8)), \
+            "a residual destination was written outside the rank's row block"
+        if count:
+            assert np.array_equal(wl.bits(r[sl]), orr), f"destination {d}: residual sum is not bit-exact"
+    if not in_place:
+        assert torch.equal(gin.host().view(torch.uint8), inp.residual.view(torch.uint8)), "the residual input was modified"
+    if count:
+        fold(stats, check_values(f64(y0[sl]), oy, inp.dtype, what=f"two-shot rank {rank}/{world} {(T, H)}"))
+    return stats
+
+
+@pytest.mark.parametrize("world,rank", [(2, 1), (4, 0), (8, 5), (16, 15)])
+@pytest.mark.parametrize("T,H", [(613, 4096), (64, 4100), (37, 20500)])
+def test_two_shot_row_blocks(world, rank, T, H):
+    stats = run_two_shot(wl.allreduce_rmsnorm_inputs(T, H, world, BF16, seed=world * 100 + rank), world, rank)
+    assert stats["max_err_ulp"] <= 2.0
+
+
+@pytest.mark.parametrize("dtype", [FP16, FP32])
+def test_two_shot_other_storage_types_and_separate_residual_input(dtype):
+    run_two_shot(wl.allreduce_rmsnorm_inputs(130, 5120, 3, dtype, seed=5), 3, 2, in_place=False)
+    run_two_shot(wl.allreduce_rmsnorm_inputs(130, 5120, 3, dtype, seed=5), 3, 1, offset=2)
+
+
+def test_two_shot_long_block_and_empty_block():
+    """A block of 4096 rows or more takes the register-capped instantiation; a rank that is dealt no
+    rows (fewer rows than ranks) launches nothing and writes nothing."""
+    run_two_shot(wl.allreduce_rmsnorm_inputs(8200, 2048, 2, BF16, seed=21), 2, 1)
+    run_two_shot(wl.allreduce_rmsnorm_inputs(3, 4096, 4, BF16, seed=22), 4, 3)
+
+
+def test_two_shot_with_single_destinations_is_the_one_shot_call_bit_for_bit():
+    inp = wl.allreduce_rmsnorm_inputs(300, 4096, 4, BF16, seed=23)
+    parts, w = [p.cuda() for p in inp.parts], inp.weight.cuda()
+    y1, r1 = torch.empty_like(parts[0]), inp.residual.cuda()
+    astra.astra_fused_allreduce_add_rmsnorm(y1, r1, parts, w, inp.eps)
+    y2, r2 = torch.empty_like(parts[0]), inp.residual.cuda()
+    astra.astra_fused_allreduce_add_rmsnorm_ex([y2], [r2], r2, parts, w, inp.eps)
+    assert torch.equal(y1, y2) and torch.equal(r1, r2)
+
+
+def test_two_shot_all_ranks_assemble_the_whole_batch():
+    """Every rank's call in turn (one GPU, so one after the other): together the row blocks fill every
+    rank's buffers with the whole batch's result (the residual exactly what the one-shot call gives)."""
+    world, T, H = 4, 1001, 4096
+    from paper_2509_07506_b200 import multi
+    inp = wl.allreduce_rmsnorm_inputs(T, H, world, BF16, seed=24)
+    parts, w = [p.cuda() for p in inp.parts], inp.weight.cuda()
+    y_ref, r_ref = torch.empty_like(parts[0]), inp.residual.cuda()
+    astra.astra_fused_allreduce_add_rmsnorm(y_ref, r_ref, parts, w, inp.eps)
+    ys = [torch.zeros_like(parts[0]) for _ in range(world)]
+    rs = [inp.residual.cuda() for _ in range(world)]      # every rank holds the residual
+    for rank in range(world):
+        first, count = multi.shard_rows(T, world, rank)
+        sl = slice(first, first + count)
+        astra.astra_fused_allreduce_add_rmsnorm_ex([y[sl] for y in ys], [r[sl] for r in rs], rs[rank][sl],
+                                                   [p[sl] for p in parts], w, inp.eps)
+    torch.cuda.synchronize()
+    # The residual is bit-exact whatever the launch shape.  y depends on the order in which a block
+    # sums the squares, which differs between the launch shape of a 250-row block and that of the
+    # 1001-row batch, so it is compared with the oracle (and across destinations bit for bit).
+    for d in range(world):
+        assert torch.equal(rs[d], r_ref) and torch.equal(ys[d], ys[0])
+    oy, orr = oracle.fused_allreduce_add_rmsnorm([wl.bits(p) for p in inp.parts], wl.bits(inp.residual),
+                                                 wl.bits(inp.weight), inp.eps, BF16, nthreads=NCPU)
+    assert np.array_equal(wl.bits(r_ref.cpu()), orr)
+    check_values(f64(ys[0].cpu()), oy, BF16, what="two-shot, assembled from four row blocks")
+    check_values(f64(y_ref.cpu()), oy, BF16, what="one-shot")
+
+
 def test_allreduce_rmsnorm_binding_refuses_bad_calls():
     e = lambda *shape: torch.zeros(shape, dtype=torch.bfloat16, device="cuda")  # noqa: E731
     with pytest.raises(ValueError):
@@ -131,6 +240,16 @@ def test_allreduce_rmsnorm_binding_refuses_bad_calls():
     y = e(4, 64)
     with pytest.raises(astra.AstraError) as err:
         astra.astra_fused_allreduce_add_rmsnorm(y, e(4, 64), [y, e(4, 64)], e(64), 1e-6)
+    assert err.value.status == 6
+    with pytest.raises(ValueError):
+        astra.astra_fused_allreduce_add_rmsnorm_ex([], [e(4, 64)], e(4, 64), [e(4, 64)], e(64), 1e-6)
+    with pytest.raises(ValueError):
+        astra.astra_fused_allreduce_add_rmsnorm_ex([e(4, 64)], [e(4, 64)] * 17, e(4, 64), [e(4, 64)], e(64), 1e-6)
+    with pytest.raises(ValueError):
+        astra.astra_fused_allreduce_add_rmsnorm_ex([e(4, 64)], [e(5, 64)], e(4, 64), [e(4, 64)], e(64), 1e-6)
+    r = e(4, 64)
+    with pytest.raises(astra.AstraError) as err:
+        astra.astra_fused_allreduce_add_rmsnorm_ex([y, y], [r], r, [e(4, 64)], e(64), 1e-6)
     assert err.value.status == 6
 
 

@@ -100,6 +100,27 @@ def _tp_worker(rank, world, port, out_dir):
         owned[sl] = 1
         dist.all_reduce(owned)
         assert bool((owned == 1).all())
+        # Two-shot form, host side: every rank's output buffer is exchanged the same way (here a file
+        # mapped by both processes stands for peer-mapped device memory), every rank stores its block
+        # into all of them, and after a barrier each rank holds the whole-batch result.
+        def export_map(arr):
+            return (rank, arr.filename)
+
+        def open_map(handle, owner):
+            assert handle[0] == owner and owner != rank
+            return np.memmap(handle[1], dtype=np.float64, mode="r+", shape=(T, H))
+
+        y_mine = np.memmap(os.path.join(out_dir, f"y{rank}.bin"), dtype=np.float64, mode="w+", shape=(T, H))
+        y_mine[:] = -1.0
+        y_mine.flush()
+        ys = multi.exchange_buffers(y_mine, export_map, open_map)
+        assert len(ys) == world and ys[rank] is y_mine
+        dist.barrier()
+        for dest in ys:
+            dest[sl] = y
+            dest.flush()
+        dist.barrier()
+        assert np.array_equal(np.asarray(y_mine), yw), "two-shot: the assembled rows differ from the whole-batch result"
         with open(os.path.join(out_dir, f"tp_ok{rank}"), "w") as fh:
             fh.write("ok")
     finally:

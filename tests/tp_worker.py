@@ -2,7 +2,8 @@
 ANOTHER PROCESS's device memory (mapped through an inter-process handle), started by
 test_gpu_allreduce.py through multi.spawn_ranks.  With one GPU in the machine both ranks use it: the
 kernel has no device-side wait, the ordering is two host barriers, so nothing here depends on the
-two ranks' kernels running at the same time.  Writes <outdir>/tp_gpu_ok<rank> on success."""
+two ranks' kernels running at the same time.  The two-shot form is checked the same way: each rank
+stores its row block into the other rank's mapped output buffers.  Writes <outdir>/tp_gpu_ok<rank> on success."""
 import os
 import sys
 
@@ -53,7 +54,21 @@ def main() -> int:
         assert np.array_equal(wl.bits(r2.cpu()), orr[sl]) and torch.equal(y2, y[sl])
         for owner in range(world):          # the mapped partials are the owners' bytes
             assert torch.equal(parts[owner].cpu(), inp.parts[owner])
-        del parts
+        # Two-shot form: every rank reduces its own row block and STORES the results into every rank's
+        # buffers (its own directly, the other rank's through the mapping).
+        y_all, r_all = torch.zeros_like(mine), inp.residual.to(dev)
+        torch.cuda.synchronize()
+        ys = multi.exchange_buffers(y_all, multi.export_cuda_tensor, multi.open_cuda_tensor)
+        rs = multi.exchange_buffers(r_all, multi.export_cuda_tensor, multi.open_cuda_tensor)
+        assert ys[rank] is y_all and rs[rank] is r_all
+        dist.barrier()                      # every buffer exists and holds its initial contents
+        astra.astra_fused_allreduce_add_rmsnorm_ex([b[sl] for b in ys], [b[sl] for b in rs], r_all[sl],
+                                                   [p[sl] for p in parts], w, inp.eps)
+        torch.cuda.synchronize()
+        dist.barrier()                      # every rank's stores have landed before anyone reads its buffers
+        assert np.array_equal(wl.bits(r_all.cpu()), orr), "two-shot: the assembled residual is not bit-exact"
+        check_values(y_all.cpu().to(torch.float64).numpy(), oy, wl.BF16, what=f"rank {rank}: two-shot y")
+        del parts, ys, rs
         dist.barrier()
         with open(os.path.join(out_dir, f"tp_gpu_ok{rank}"), "w") as fh:
             fh.write("ok")
