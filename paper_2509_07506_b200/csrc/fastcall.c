@@ -154,6 +154,10 @@ static PyObject *fc_launch(PyObject *self, PyObject *const *args, Py_ssize_t nar
     if (stream == NULL && PyErr_Occurred()) return NULL;
     const astra_dtype_t dt = (astra_dtype_t)p->dtype;
     void *fn = entry_points[p->kind];
+    if (fn == NULL) {  /* unbound again since the call was prepared */
+        PyErr_SetString(PyExc_RuntimeError, "no entry point bound for this kind of call");
+        return NULL;
+    }
     astra_status_t st;
     switch (p->kind) {
         case KIND_RMSNORM:
