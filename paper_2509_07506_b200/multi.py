@@ -154,3 +154,54 @@ def open_cuda_tensor(handle, owner: int) -> torch.Tensor:
     tensor over it (no copy).  Reading it is ordinary device memory access through the mapping."""
     rebuild, args = handle
     return rebuild(*args)
+
+
+class PeerEvents:
+    """Stream ordering between the ranks of one node without synchronising any host with its GPU.
+
+    The fused all-reduce kernels wait for nothing on the device; the caller must order them after
+    every rank's partial has been written (and, in the two-shot form, order the consumers after every
+    rank's stores).  Each rank owns one inter-process CUDA event; the handles are exchanged once.
+    A phase then goes: every rank enqueues its producer work and calls ``record()``; the ranks meet
+    at a host barrier (``barrier()``: hosts only, the GPUs keep running); every rank calls
+    ``wait_for_all()``, which makes its stream wait for all ranks' recorded events, and enqueues the
+    consumer.  The host barrier is what guarantees that each ``wait_for_all`` sees the peers' events
+    already recorded: a stream wait on an event captures the event's most recent record at the time
+    of the call, and a wait on an event that was never recorded returns at once.  Nothing here spins
+    on the device: the waits are stream dependencies resolved by the driver."""
+
+    def __init__(self, device: torch.device, group=None):
+        self.device = device
+        self.group = group
+        self.mine = torch.cuda.Event(enable_timing=False, interprocess=True)
+        if dist.is_available() and dist.is_initialized():
+            self.rank, world = dist.get_rank(group), dist.get_world_size(group)
+            with torch.cuda.device(device):
+                handle = self.mine.ipc_handle()
+            handles = [None] * world
+            dist.all_gather_object(handles, handle, group=group)
+            self.events = [self.mine if owner == self.rank else torch.cuda.Event.from_ipc_handle(device, handles[owner])
+                           for owner in range(world)]
+        else:
+            self.rank, self.events = 0, [self.mine]
+
+    def record(self, stream: torch.cuda.Stream | None = None) -> None:
+        """Mark the point in `stream` (default: the current stream) that the peers will wait for."""
+        self.mine.record(stream if stream is not None else torch.cuda.current_stream(self.device))
+
+    def barrier(self) -> None:
+        """Host-only meeting point between ``record`` and ``wait_for_all`` (no GPU synchronisation)."""
+        if dist.is_available() and dist.is_initialized():
+            dist.barrier(group=self.group)
+
+    def wait_for_all(self, stream: torch.cuda.Stream | None = None) -> None:
+        """Order everything enqueued on `stream` from here on after every rank's recorded event."""
+        stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+        for ev in self.events:
+            stream.wait_event(ev)
+
+    def phase(self, stream: torch.cuda.Stream | None = None) -> None:
+        """record, host barrier, wait for all: one complete ordering step."""
+        self.record(stream)
+        self.barrier()
+        self.wait_for_all(stream)

@@ -68,7 +68,27 @@ def main() -> int:
         dist.barrier()                      # every rank's stores have landed before anyone reads its buffers
         assert np.array_equal(wl.bits(r_all.cpu()), orr), "two-shot: the assembled residual is not bit-exact"
         check_values(y_all.cpu().to(torch.float64).numpy(), oy, wl.BF16, what=f"rank {rank}: two-shot y")
-        del parts, ys, rs
+        # The same two steps ordered by inter-process events instead of host synchronisation: the
+        # partial is produced by a kernel on the stream, the ranks' streams wait for one another's
+        # events, and no host waits for its GPU until the results are read back.
+        ev_written, ev_read = multi.PeerEvents(dev), multi.PeerEvents(dev)
+        for rep in range(3):
+            # new partials every repetition (the oracle gets the same bits): a stale read would show
+            scaled = [(p.to(torch.float32) * float(rep + 2)).to(p.dtype) for p in inp.parts]
+            mine.copy_(scaled[rank])
+            r_all.copy_(inp.residual)
+            y_all.zero_()
+            ev_written.phase()              # every rank's partial (and reset buffers) precede every rank's kernel
+            astra.astra_fused_allreduce_add_rmsnorm_ex([b[sl] for b in ys], [b[sl] for b in rs], r_all[sl],
+                                                       [p[sl] for p in parts], w, inp.eps)
+            ev_read.phase()                 # every rank's kernel precedes any reuse of partials and any read of results
+            got_y, got_r = y_all.cpu(), r_all.cpu()      # stream-ordered copies: they follow the waits above
+            oy3, orr3 = oracle.fused_allreduce_add_rmsnorm([wl.bits(p) for p in scaled], wl.bits(inp.residual),
+                                                           wl.bits(inp.weight), inp.eps, wl.BF16, nthreads=4)
+            assert np.array_equal(wl.bits(got_r), orr3), f"event-ordered two-shot, repetition {rep}: residual not bit-exact"
+            check_values(got_y.to(torch.float64).numpy(), oy3, wl.BF16, what=f"rank {rank}: event-ordered two-shot y")
+        torch.cuda.synchronize()
+        del parts, ys, rs, ev_written, ev_read
         dist.barrier()
         with open(os.path.join(out_dir, f"tp_gpu_ok{rank}"), "w") as fh:
             fh.write("ok")
