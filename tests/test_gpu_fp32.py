@@ -21,6 +21,13 @@ def test_rmsnorm_fp32(T, H):
     run_rmsnorm(wl.rmsnorm_inputs(T, H, FP32, eps=1e-5, seed=H))
 
 
+@pytest.mark.parametrize("T,H", [(1100, 4096), (1024, 2048), (1500, 1024), (700, 4096)])
+def test_rmsnorm_fp32_streaming_sizes(T, H):
+    """More rows than one wave of blocks: 32-byte vectors (two per thread) where the rows allow it,
+    16-byte vectors otherwise; every row against the oracle."""
+    run_rmsnorm(wl.rmsnorm_inputs(T, H, FP32, eps=1e-5, seed=T))
+
+
 @pytest.mark.parametrize("offset", [1, 2, 4])
 def test_rmsnorm_fp32_pointer_offsets(offset):
     run_rmsnorm(wl.rmsnorm_inputs(7, 4096, FP32, eps=1e-6, seed=offset), offset=offset)

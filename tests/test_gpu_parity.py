@@ -202,6 +202,15 @@ def test_rmsnorm_pointer_offsets(offset, H):
     run_rmsnorm(wl.rmsnorm_inputs(7, H, BF16, eps=1e-6, seed=offset), offset=offset)
 
 
+@pytest.mark.parametrize("offset", [0, 8, 16, 4])
+@pytest.mark.parametrize("T,H", [(1033, 4096), (1024, 5120), (1100, 2048), (333, 4096)])
+def test_rmsnorm_streaming_alignments(offset, T, H):
+    """From 1024 rows on, rows that are 32-byte aligned take two 32-byte vectors per thread, 16-byte
+    aligned ones (offset 8) four 16-byte vectors, 8-byte aligned ones (offset 4) 8-byte vectors; between
+    one wave of rows and 1024 rows the 16-byte form serves both."""
+    run_rmsnorm(wl.rmsnorm_inputs(T, H, BF16, eps=1e-5, seed=offset + T), offset=offset)
+
+
 def test_rmsnorm_closed_forms_on_gpu():
     # constant row -> sign(c) * w ; zero row -> 0
     H = 4096
