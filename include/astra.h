@@ -170,8 +170,8 @@ astra_status_t astra_merge_attn_states_lse_ex(void *v_out, float *lse_out,
  *   x_parts  HOST array of n_parts device pointers, in rank order, each a dense [T, H] tensor.
  *            A partial may live in another GPU's memory if that memory is mapped into this
  *            process (peer access): the kernel reads it with ordinary per-thread loads only.
- *   n_parts  1 .. 16 (else ASTRA_ERR_BAD_SHAPE).  n_parts = 1 computes exactly what
- *            astra_fused_add_rmsnorm_ex computes with separate y.
+ *   n_parts  1 .. 16 (else ASTRA_ERR_BAD_SHAPE).  n_parts = 1 is the operation of
+ *            astra_fused_add_rmsnorm_ex with separate y (same residual bits; y by the same arithmetic).
  *   weight   [H].
  *
  * Arithmetic: every addition is one binary32 addition; the partials are added in rank order

@@ -35,6 +35,11 @@ const char kBuildId[] = "astra-build-id:" ASTRA_BUILD_ID;
 // [1024, 14336] = 7168 blocks, 0.5 % at [4096, 14336], 1.6 % slower at [8192, 14336] = 57344 blocks);
 // below it the inputs are requested ahead of the dependency wait.
 constexpr uint32_t kSiluPrefetchMaxBlocks = 1u << 14;
+// Range of grid sizes (in 256-thread blocks of one 32-byte vector per thread) in which the 32-byte
+// form is used: from 640 blocks (measured: slower at 448, faster at 896) to 8192 (faster at 7168,
+// slower at 14336).
+constexpr int64_t kSiluWideMinBlocks = 640;
+constexpr int64_t kSiluWideMaxBlocks = 8192;
 
 template <int DT, int UVEC, int UNROLL, int THREADS>
 cudaError_t launch_silu(uint16_t *out, const uint16_t *gate, const uint16_t *up, int64_t T, int64_t D,
@@ -50,7 +55,7 @@ cudaError_t launch_silu(uint16_t *out, const uint16_t *gate, const uint16_t *up,
         const uint32_t blocks = (total + tile - 1) / tile;
         const FastDiv per_row = FastDiv::make(static_cast<uint32_t>(nvec));
         cudaError_t err;
-        if (UVEC == 8 && blocks <= kSiluPrefetchMaxBlocks)
+        if (UVEC >= 8 && blocks <= kSiluPrefetchMaxBlocks)
             err = launch(silu_and_mul_kernel<DT, VEC, UNROLL, THREADS, Ld::StreamReadOnly, St::Stream, THREADS * UNROLL>,
                          blocks, THREADS, stream, out + t0 * out_pitch, gate + t0 * gate_pitch, up + t0 * up_pitch,
                          total, per_row, out_pitch, gate_pitch, up_pitch);
@@ -67,10 +72,21 @@ cudaError_t launch_silu(uint16_t *out, const uint16_t *gate, const uint16_t *up,
 template <int DT>
 cudaError_t dispatch_silu(uint16_t *out, const uint16_t *gate, const uint16_t *up, int64_t T, int64_t D,
                    int64_t out_pitch, int64_t gate_pitch, int64_t up_pitch, cudaStream_t stream) {
-    const int vec = VecPick(8).extent(D).extent(out_pitch).extent(gate_pitch).extent(up_pitch)
-                        .pointer(out).pointer(gate).pointer(up).vec;
+    int vec = VecPick(16).extent(D).extent(out_pitch).extent(gate_pitch).extent(up_pitch)
+                  .pointer(out).pointer(gate).pointer(up).vec;
     // One 16-byte vector per thread and 256-thread blocks: the smallest work quantum that still
     // keeps the block scheduler ahead, which gives the shortest drain at the end of the grid.
+    // Between about one and ten waves of blocks, one 32-byte vector per thread (half as many blocks,
+    // each still prefetching its share ahead of the dependency wait) is faster where everything is
+    // 32-byte aligned: 4.21 -> 3.83 us at [256, 14336], 7.19 -> 6.73 us at [512, 14336], 13.2 -> 12.6 us
+    // at [1024, 14336], 25.2 -> 24.8 us at [2048, 14336] (L2-cold, bf16); it is slower below that
+    // (2.56 -> 3.14 us at [128, 14336]) and above it (98.3 -> 99.9 us at [8192, 14336]).
+    if (vec == 16) {
+        const int64_t blocks_wide = (T * (D / 16) + 255) / 256;
+        if (blocks_wide >= kSiluWideMinBlocks && blocks_wide <= kSiluWideMaxBlocks)
+            return launch_silu<DT, 16, 1, 256>(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, stream);
+        vec = 8;  // everything that is 32-byte aligned is 16-byte aligned
+    }
     switch (vec) {
         case 8: return launch_silu<DT, 8, 1, 256>(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, stream);
         case 4: return launch_silu<DT, 4, 4, 256>(out, gate, up, T, D, out_pitch, gate_pitch, up_pitch, stream);

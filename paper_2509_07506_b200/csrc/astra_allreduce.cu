@@ -14,7 +14,7 @@ using namespace astra::host;
 
 inline int round_up_to(int v, int m) { return (v + m - 1) / m * m; }
 
-// Register-resident rows hold at most 32 16-bit units per thread in vectors of 8 or 16 bytes.
+// Register-resident rows hold at most 32 16-bit units per thread in vectors of 8, 16 or 32 bytes.
 // UVEC is the vector width in units, VPT the vectors per thread.
 // `dense` selects the instantiation whose registers are capped so that five 256-thread blocks fit an
 // SM; it exists for the streaming shape (two loads in flight, 16 units per thread) only.
@@ -120,14 +120,48 @@ cudaError_t choose_shape(const AllreduceOperands &op, const uint16_t *w, int64_t
   return cudaErrorInvalidValue;
 }
 
+// Streaming sizes whose operands are 32-byte aligned throughout: 32-byte accesses, 16 units per thread
+// in one vector (256-thread blocks at H = 4096, 55 registers uncapped; capping them lost here), two
+// partial loads in flight, four from four partials on (71 registers).  Measured L2-cold against the
+// 16-byte form at [8192, 4096]: 50.6 -> 49.2 us with 2 partials, 70.8 -> 66.6 us with 4, 110.9 -> 104.7 us
+// with 8; at [1024, 4096]: 8.3 -> 7.7, 10.9 -> 10.3, 16.2 -> 15.9 us.  Returns false where the form does
+// not apply (rows too narrow for 128-thread blocks or too wide for the registers).
+constexpr int kWideStreamGroup = 4;
+
+template <int DT>
+bool launch_wide(const AllreduceOperands &op, const uint16_t *w, int64_t T, int H, float eps, cudaStream_t stream,
+                 cudaError_t *err) {
+    constexpr int UVEC = 16;
+    const int nvec = H / (UVEC / Storage<DT>::UNITS);
+    int threads = 0;
+    if (op.n_parts >= kWideStreamGroup) {
+        const int vpt = pick_vpt<UVEC, kWideStreamGroup>(nvec, 16, &threads);
+        if (vpt > 0 && threads >= 128) {
+            *err = launch_rows<DT, UVEC, kWideStreamGroup>(op, w, T, H, eps, vpt, threads, stream);
+            return true;
+        }
+    }
+    const int vpt = pick_vpt<UVEC, kStreamGroup>(nvec, 16, &threads);
+    if (vpt > 0 && threads >= 128) {
+        *err = launch_rows<DT, UVEC, kStreamGroup>(op, w, T, H, eps, vpt, threads, stream);
+        return true;
+    }
+    return false;
+}
+
 template <int DT>
 cudaError_t dispatch(const AllreduceOperands &op, const uint16_t *w, int64_t T, int H, float eps,
                      cudaStream_t stream) {
-    VecPick pick(8);
+    VecPick pick(16);
     pick.extent(static_cast<int64_t>(H) * Storage<DT>::UNITS).pointer(op.r).pointer(w);
     for (int p = 0; p < op.n_parts; ++p) pick.pointer(op.part[p]);
     for (int d = 0; d < op.n_y; ++d) pick.pointer(op.y_out[d]);
     for (int d = 0; d < op.n_r; ++d) pick.pointer(op.r_out[d]);
+    if (pick.vec == 16) {
+        cudaError_t err = cudaSuccess;
+        if (T > kLatencyRows && launch_wide<DT>(op, w, T, H, eps, stream, &err)) return err;
+        pick.vec = 8;  // everything that is 32-byte aligned is 16-byte aligned
+    }
     switch (pick.vec) {
         case 8: return choose_shape<DT, 8>(op, w, T, H, eps, stream);
         case 4: return choose_shape<DT, 4>(op, w, T, H, eps, stream);

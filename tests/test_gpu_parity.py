@@ -239,6 +239,16 @@ def test_silu_widths(dtype, D):
     run_silu(wl.silu_inputs(5, D, dtype, std=2.0, seed=D))
 
 
+@pytest.mark.parametrize("dtype", [BF16, FP16])
+@pytest.mark.parametrize("T,D,offset", [(256, 14336, 0), (1024, 4096, 0), (700, 5120, 16), (700, 5120, 8), (2048, 14336, 0),
+                                        (300, 11008, 0)])
+def test_silu_mid_sizes(dtype, T, D, offset):
+    """Between about one and ten waves of blocks the 32-byte-vector form runs where gate, up and out are
+    32-byte aligned (offsets 0 and 16; D = 11008 puts the up half only 16-byte aligned), the 16-byte
+    form otherwise."""
+    run_silu(wl.silu_inputs(T, D, dtype, std=2.0, seed=T + D), offset=offset)
+
+
 @pytest.mark.parametrize("offset", [1, 2, 4])
 def test_silu_pointer_offsets(offset):
     run_silu(wl.silu_inputs(9, 4096, BF16, seed=offset), offset=offset)

@@ -91,6 +91,24 @@ def test_silu_ex_separate_gate_and_up(dtype, D, pitch, col0):
     assert torch.equal(gv.cpu(), gate_h) and torch.equal(uv.cpu(), up_h)
 
 
+def test_silu_ex_mid_size_pitched_rows():
+    """Enough rows for the 32-byte-vector form, with pitches (multiples of 16 elements) that keep every
+    row 32-byte aligned, and with a pitch that leaves rows only 16-byte aligned."""
+    T, D = 600, 5120
+    inp = wl.silu_inputs(T, D, BF16, std=2.0, seed=77)
+    gate_h, up_h = inp.input[:, :D].contiguous(), inp.input[:, D:].contiguous()
+    want = oracle.silu_and_mul(wl.bits(inp.input), BF16)
+    for pitch in (D + 64, D + 8):
+        gb, gv = pitched(gate_h, pitch, 0)
+        ub, uv = pitched(up_h, pitch + 16, 0)
+        ob, ov = pitched(torch.zeros_like(gate_h), pitch + 32, 0)
+        astra.astra_silu_and_mul_ex(ov, gv, uv)
+        torch.cuda.synchronize()
+        check_values(f64(ov.cpu()), want, BF16, what=f"silu_ex mid size, pitch {pitch}")
+        for buf in (gb, ub, ob):
+            assert untouched(buf, 0, D)
+
+
 def test_silu_ex_on_packed_rows_equals_plain_call():
     inp = wl.silu_inputs(64, 14336, BF16, seed=4)
     d = inp.input.cuda()
