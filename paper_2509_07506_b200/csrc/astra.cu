@@ -320,7 +320,10 @@ cudaError_t launch_rmsnorm(RmsnormOperands op, const uint16_t *w, int64_t T, int
 // Measured L2-cold against the 16-byte form, bf16: 11.36 -> 11.08 us at [2048, 4096], 40.3 -> 39.8 us at
 // [8192, 4096], 13.7 -> 13.5 / 50.1 -> 49.6 us at [2048 / 8192, 5120], 0.2-0.4 % at H = 8192, 6.48 -> 6.39 us
 // at [1024, 4096]; 1-2 % slower at [512, 5120] and [512, 8192] and no different at or below one wave of
-// rows, so the 16-byte forms stay below 1024 rows.
+// rows, so the 16-byte forms stay below 1024 rows.  Blocks of 64 to 448 threads, i.e. H = 2048 ... 14336
+// for the 16-bit types (also measured: 21.4 -> 20.6 us at [8192, 2048], 104.4 -> 103.9 us at
+// [8192, 11008], 136.7 -> 135.8 us at [8192, 14336], 18.7 -> 18.4 us at [1024, 14336]); wider rows would
+// leave one 512-thread block per SM and keep 16 units per thread at full occupancy instead.
 constexpr int64_t kWideVectorRows = 1024;
 template <int DT>
 bool launch_rmsnorm_wide(const RmsnormOperands &op, const uint16_t *w, int64_t T, int H, float eps,
@@ -328,7 +331,7 @@ bool launch_rmsnorm_wide(const RmsnormOperands &op, const uint16_t *w, int64_t T
     constexpr int UVEC = 16, VEC = UVEC / Storage<DT>::UNITS, VPT = 2;
     const int nvec = H / VEC;
     const int threads = round_up((nvec + VPT - 1) / VPT, 32);
-    if (T < kWideVectorRows || threads < 128 || threads > 256) return false;
+    if (T < kWideVectorRows || threads < 64 || threads > 448) return false;
     const float inv_H = 1.0f / static_cast<float>(H);
     *err = cudaSuccess;
     for (int64_t t0 = 0; t0 < T && *err == cudaSuccess; t0 += kMaxGridX) {

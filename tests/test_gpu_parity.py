@@ -203,7 +203,8 @@ def test_rmsnorm_pointer_offsets(offset, H):
 
 
 @pytest.mark.parametrize("offset", [0, 8, 16, 4])
-@pytest.mark.parametrize("T,H", [(1033, 4096), (1024, 5120), (1100, 2048), (333, 4096)])
+@pytest.mark.parametrize("T,H", [(1033, 4096), (1024, 5120), (1100, 2048), (333, 4096), (1025, 14336), (1030, 11008),
+                                 (1024, 16384), (1040, 1024)])
 def test_rmsnorm_streaming_alignments(offset, T, H):
     """From 1024 rows on, rows that are 32-byte aligned take two 32-byte vectors per thread, 16-byte
     aligned ones (offset 8) four 16-byte vectors, 8-byte aligned ones (offset 4) 8-byte vectors; between
