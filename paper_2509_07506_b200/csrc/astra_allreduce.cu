@@ -135,7 +135,15 @@ bool launch_wide(const AllreduceOperands &op, const uint16_t *w, int64_t T, int 
     const int nvec = H / (UVEC / Storage<DT>::UNITS);
     int threads = 0;
     if (op.n_parts >= kWideStreamGroup) {
-        const int vpt = pick_vpt<UVEC, kWideStreamGroup>(nvec, 16, &threads);
+        int vpt = pick_vpt<UVEC, kWideStreamGroup>(nvec, 16, &threads);
+        // With four loads in flight a thread needs 71 registers: above 384 threads only one block would
+        // fit an SM.  Two vectors per thread in blocks half the size (126 registers, two blocks per SM)
+        // keep as many threads resident with twice the bytes in flight each: at [4096, 8192], 78.8 ->
+        // 68.0 us with 4 partials and 117.3 -> 105.6 us with 8.
+        if (vpt == 1 && threads > 384) {
+            vpt = 2;
+            threads = round_up_to((nvec + 1) / 2, 32);
+        }
         if (vpt > 0 && threads >= 128) {
             *err = launch_rows<DT, UVEC, kWideStreamGroup>(op, w, T, H, eps, vpt, threads, stream);
             return true;
