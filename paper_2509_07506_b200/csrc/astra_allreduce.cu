@@ -120,41 +120,58 @@ cudaError_t choose_shape(const AllreduceOperands &op, const uint16_t *w, int64_t
   return cudaErrorInvalidValue;
 }
 
-// Streaming sizes whose operands are 32-byte aligned throughout: 32-byte accesses, 16 units per thread
-// in one vector (256-thread blocks at H = 4096, 55 registers uncapped; capping them lost here), two
-// partial loads in flight, four from four partials on (71 registers).  Measured L2-cold against the
-// 16-byte form at [8192, 4096]: 50.6 -> 49.2 us with 2 partials, 70.8 -> 66.6 us with 4, 110.9 -> 104.7 us
-// with 8; at [1024, 4096]: 8.3 -> 7.7, 10.9 -> 10.3, 16.2 -> 15.9 us.  Returns false where the form does
-// not apply (rows too narrow for 128-thread blocks or too wide for the registers).
-constexpr int kWideStreamGroup = 4;
+// Streaming sizes whose operands are 32-byte aligned throughout: 32-byte accesses.  Measured L2-cold
+// against the 16-byte form at [8192, 4096]: 50.6 -> 49.2 us with 2 partials, 70.8 -> 66.6 us with 4,
+// 110.9 -> 104.7 us with 8; at [1024, 4096]: 8.3 -> 7.7, 10.9 -> 10.3, 16.2 -> 15.9 us.
+//
+// Four shapes: one or two vectors per thread (16 or 32 units), two or four partial loads in flight
+// (four only from four partials on).  What decides between them is how many bytes of loads an SM has
+// in flight, i.e. resident blocks x threads x bytes per thread, with the resident blocks set by the
+// registers (56 / 96 / 72 / 128 per thread as compiled for sm_100a, allocated in eights, 65536 per
+// SM).  The measurements across H = 2048 ... 16384 fit one rule: take the first shape, in the order
+// below, that keeps about 90 KB in flight per SM; if none does, the one with the most.  Examples:
+// H = 4096 takes one vector and four in flight (three 256-thread blocks per SM); H = 8192 with four
+// in flight would leave one 512-thread block per SM, so it takes two vectors in 256-thread blocks
+// (78.8 -> 68.0 us with 4 partials, 117.3 -> 105.6 us with 8); H = 10240 with two in flight takes two
+// vectors in 320-thread blocks (two per SM) rather than one 640-thread block (61.6 against 76.7 us);
+// H = 16384 takes one vector in one 1024-thread block (143.1 against 155.8 us with 4 partials).
+// Returns false where no shape applies (rows too narrow for 128-thread blocks, or too wide).
+struct WideShape {
+    int vpt, group, regs, max_threads, min_threads;
+};
+constexpr WideShape kWideShapes[] = {
+    {1, 4, 72, 512, 128}, {2, 4, 128, 256, 64}, {1, 2, 56, 1024, 128}, {2, 2, 96, 512, 64}};
+constexpr int64_t kWideBytesInFlight = 90 * 1024;
 
 template <int DT>
 bool launch_wide(const AllreduceOperands &op, const uint16_t *w, int64_t T, int H, float eps, cudaStream_t stream,
                  cudaError_t *err) {
     constexpr int UVEC = 16;
     const int nvec = H / (UVEC / Storage<DT>::UNITS);
-    int threads = 0;
-    if (op.n_parts >= kWideStreamGroup) {
-        int vpt = pick_vpt<UVEC, kWideStreamGroup>(nvec, 16, &threads);
-        // With four loads in flight a thread needs 71 registers: above 384 threads only one block would
-        // fit an SM.  Two vectors per thread in blocks half the size (126 registers, two blocks per SM)
-        // keep as many threads resident with twice the bytes in flight each: at [4096, 8192], 78.8 ->
-        // 68.0 us with 4 partials and 117.3 -> 105.6 us with 8.
-        if (vpt == 1 && threads > 384) {
-            vpt = 2;
-            threads = round_up_to((nvec + 1) / 2, 32);
+    int best = -1, best_threads = 0;
+    int64_t best_bytes = 0;
+    for (int c = 0; c < 4; ++c) {
+        const WideShape &sh = kWideShapes[c];
+        if (sh.group > kStreamGroup && op.n_parts < sh.group) continue;
+        const int threads = round_up_to((nvec + sh.vpt - 1) / sh.vpt, 32);
+        if (threads > sh.max_threads || threads < sh.min_threads) continue;
+        const int by_regs = 65536 / (sh.regs * threads), by_threads = 2048 / threads;
+        const int blocks = by_regs < by_threads ? by_regs : by_threads;
+        const int64_t bytes = static_cast<int64_t>(blocks) * threads * sh.vpt * (sh.group + 1) * 32;
+        if (bytes > best_bytes) {
+            best = c;
+            best_bytes = bytes;
+            best_threads = threads;
         }
-        if (vpt > 0 && threads >= 128) {
-            *err = launch_rows<DT, UVEC, kWideStreamGroup>(op, w, T, H, eps, vpt, threads, stream);
-            return true;
-        }
+        if (bytes >= kWideBytesInFlight) break;  // the first shape that reaches it is also the largest so far
     }
-    const int vpt = pick_vpt<UVEC, kStreamGroup>(nvec, 16, &threads);
-    if (vpt > 0 && threads >= 128) {
-        *err = launch_rows<DT, UVEC, kStreamGroup>(op, w, T, H, eps, vpt, threads, stream);
-        return true;
-    }
-    return false;
+    if (best < 0) return false;
+    const WideShape &sh = kWideShapes[best];
+    if (sh.group == 4)
+        *err = launch_rows<DT, UVEC, 4>(op, w, T, H, eps, sh.vpt, best_threads, stream);
+    else
+        *err = launch_rows<DT, UVEC, kStreamGroup>(op, w, T, H, eps, sh.vpt, best_threads, stream);
+    return true;
 }
 
 template <int DT>
