@@ -228,8 +228,14 @@ inline unsigned grid_for(int64_t work) {
 
 template <typename... KArgs, typename... Args>
 inline astra_status_t run(void (*kernel)(KArgs...), unsigned grid, cudaStream_t stream, Args... args) {
-    kernel<<<grid, kBlock, 0, stream>>>(static_cast<KArgs>(args)...);
-    return cudaGetLastError() == cudaSuccess ? ASTRA_OK : ASTRA_ERR_CUDA;
+    // the launch's own return value: an error some other code left pending is neither read nor cleared
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kBlock);
+    cfg.stream = stream;
+    if (cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...) == cudaSuccess) return ASTRA_OK;
+    (void)cudaGetLastError();  // the refusal has been reported through the status
+    return ASTRA_ERR_CUDA;
 }
 
 // Runs CALL with DT bound to the (validated, 16-bit) dtype and VARIANT to the design.
