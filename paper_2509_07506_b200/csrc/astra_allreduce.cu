@@ -33,7 +33,9 @@ cudaError_t launch_reg(const AllreduceOperands &op, const uint16_t *w, unsigned 
     return cudaErrorInvalidValue;
 }
 
-// Two launch shapes, chosen by the number of rows (measured at H = 4096 with 2, 4 and 8 partials):
+// Launch shapes of the 16-byte forms (operands that are not 32-byte aligned throughout; the 32-byte
+// forms further down serve everything else, at every row count), chosen by the number of rows
+// (measured at H = 4096 with 2, 4 and 8 partials):
 //  - streaming (more rows than one wave of blocks holds): two partial loads in flight per vector
 //    position and 16 units per thread (256-thread blocks at H = 4096).  It beat four and eight in
 //    flight and every other per-thread share by 3 to 25 % at [1024, 4096] and [8192, 4096]: the
@@ -44,7 +46,10 @@ cudaError_t launch_reg(const AllreduceOperands &op, const uint16_t *w, unsigned 
 //    partials the queue stays at two, the per-thread share is still 8 units: 1.8 against 2.0 us).
 constexpr int kStreamGroup = 2;
 constexpr int kLatencyGroup = 8;
-constexpr int64_t kLatencyRows = 2 * 148;  // two 512-thread blocks per SM on the 148 SMs of a B200
+#ifndef ASTRA_ALLREDUCE_LATENCY_ROWS
+#define ASTRA_ALLREDUCE_LATENCY_ROWS (2 * 148)
+#endif
+constexpr int64_t kLatencyRows = ASTRA_ALLREDUCE_LATENCY_ROWS;  // two 512-thread blocks per SM on the 148 SMs of a B200
 // From this many rows on the streaming shape runs in its register-capped form (five resident blocks
 // per SM instead of four): 1-2 % faster at [8192, 4096], neutral to 3 % slower at [1024, 4096].
 constexpr int64_t kDenseRows = 4096;
@@ -139,6 +144,10 @@ cudaError_t choose_shape(const AllreduceOperands &op, const uint16_t *w, int64_t
 struct WideShape {
     int vpt, group, regs, max_threads, min_threads;
 };
+#ifndef ASTRA_ALLREDUCE_DEEP_QUEUE_ROWS
+#define ASTRA_ALLREDUCE_DEEP_QUEUE_ROWS 128
+#endif
+constexpr int64_t kDeepQueueRows = ASTRA_ALLREDUCE_DEEP_QUEUE_ROWS;
 constexpr WideShape kWideShapes[] = {
     {1, 4, 72, 512, 128}, {2, 4, 128, 256, 64}, {1, 2, 56, 1024, 128}, {2, 2, 96, 512, 64}};
 constexpr int64_t kWideBytesInFlight = 90 * 1024;
@@ -148,6 +157,19 @@ bool launch_wide(const AllreduceOperands &op, const uint16_t *w, int64_t T, int 
                  cudaError_t *err) {
     constexpr int UVEC = 16;
     const int nvec = H / (UVEC / Storage<DT>::UNITS);
+    // Few rows and more than four partials: all of a row's partials in one round trip (eight loads in
+    // flight, one vector per thread); with so few blocks the registers that costs do not matter.
+    // Device time from a graph, 8 partials, against the streaming shapes: 3.19 -> 2.70 us at [16, 4096],
+    // 4.17 -> 3.41 us at [16, 8192], 4.12 -> 3.85 us at [128, 4096]; slower from 192 rows on (7.93 -> 8.89 us
+    // at [192, 8192]).  With up to four partials the streaming shapes are the fastest at every row
+    // count (1.65 / 1.98 us at [16, 4096] with 2 / 4 partials, where the 16-byte shapes took 2.08 / 2.40).
+    if (T <= kDeepQueueRows && op.n_parts > 4) {
+        const int threads = round_up_to(nvec, 32);
+        if (threads >= 128 && threads <= allreduce_reg_max_threads(16, kLatencyGroup)) {
+            *err = launch_rows<DT, UVEC, kLatencyGroup>(op, w, T, H, eps, 1, threads, stream);
+            return true;
+        }
+    }
     int best = -1, best_threads = 0;
     int64_t best_bytes = 0;
     for (int c = 0; c < 4; ++c) {
@@ -184,7 +206,7 @@ cudaError_t dispatch(const AllreduceOperands &op, const uint16_t *w, int64_t T, 
     for (int d = 0; d < op.n_r; ++d) pick.pointer(op.r_out[d]);
     if (pick.vec == 16) {
         cudaError_t err = cudaSuccess;
-        if (T > kLatencyRows && launch_wide<DT>(op, w, T, H, eps, stream, &err)) return err;
+        if (launch_wide<DT>(op, w, T, H, eps, stream, &err)) return err;
         pick.vec = 8;  // everything that is 32-byte aligned is 16-byte aligned
     }
     switch (pick.vec) {

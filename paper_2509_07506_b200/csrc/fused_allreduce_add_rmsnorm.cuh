@@ -75,7 +75,7 @@ __device__ __forceinline__ void accumulate(float (&s)[VEC], const float (&x)[VEC
 // thread beat two vectors per thread in half as many threads by 3 to 9 % (e.g. 157.9 -> 143.1 us at
 // [4096, 16384] with 4 partials, 82.2 -> 77.4 us at [4096, 11008] with 2).
 __host__ __device__ constexpr int allreduce_reg_max_threads(int units, int group) {
-    return group > 4 ? (units <= 8 ? 512 : (units <= 16 ? 256 : 128))
+    return group > 4 ? (units <= 16 ? 512 : 128)
          : group > 2 ? (units <= 8 ? 1024 : (units <= 16 ? 512 : 256))
                      : (units <= 16 ? 1024 : 512);
 }
