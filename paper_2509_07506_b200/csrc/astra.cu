@@ -324,14 +324,22 @@ cudaError_t launch_rmsnorm(RmsnormOperands op, const uint16_t *w, int64_t T, int
 // for the 16-bit types (also measured: 21.4 -> 20.6 us at [8192, 2048], 104.4 -> 103.9 us at
 // [8192, 11008], 136.7 -> 135.8 us at [8192, 14336], 18.7 -> 18.4 us at [1024, 14336]); wider rows would
 // leave one 512-thread block per SM and keep 16 units per thread at full occupancy instead.
-constexpr int64_t kWideVectorRows = 1024;
+// The same form also wins at decode sizes, where its blocks of half as many warps start and reduce
+// faster (device time from a graph, bf16: 1.61 -> 1.39 us at [1, 4096], 1.70 -> 1.49 us at [16, 4096],
+// 2.09 -> 1.87 us at [16, 8192], 1.58 -> 1.45 us at [16, 2048]); at 64 to 768 rows it is level or slower
+// (1.77 -> 1.94 us at [64, 4096], 3.38 -> 3.53 us at [256, 8192]).
+constexpr int64_t kWideVectorDecodeRows = 16;
+#ifndef ASTRA_RMSNORM_WIDE_VECTOR_ROWS
+#define ASTRA_RMSNORM_WIDE_VECTOR_ROWS 1024
+#endif
+constexpr int64_t kWideVectorRows = ASTRA_RMSNORM_WIDE_VECTOR_ROWS;
 template <int DT>
 bool launch_rmsnorm_wide(const RmsnormOperands &op, const uint16_t *w, int64_t T, int H, float eps,
                          cudaStream_t stream, cudaError_t *err) {
     constexpr int UVEC = 16, VEC = UVEC / Storage<DT>::UNITS, VPT = 2;
     const int nvec = H / VEC;
     const int threads = round_up((nvec + VPT - 1) / VPT, 32);
-    if (T < kWideVectorRows || threads < 64 || threads > 448) return false;
+    if ((T > kWideVectorDecodeRows && T < kWideVectorRows) || threads < 64 || threads > 448) return false;
     const float inv_H = 1.0f / static_cast<float>(H);
     *err = cudaSuccess;
     for (int64_t t0 = 0; t0 < T && *err == cudaSuccess; t0 += kMaxGridX) {
